@@ -1,0 +1,157 @@
+/*
+ * modse.h - C ABI of the MoDSE (Mixture of Diverse Size Experts) feed-forward
+ * layer for NVIDIA B200 (sm_100a).
+ *
+ * The layer is the one of "Mixture of Diverse Size Experts" (arXiv 2409.12210):
+ *   gate     G(x) = Softmax(KeepTopK(H(x), k)),  H(x) = x . W_g      (Sec. 2, Eq. 2-3)
+ *   output   y    = sum_i G_i(x) E_i(x)                               (Sec. 3.1, Eq. 4)
+ * where expert E_i is a bias-free SwiGLU feed-forward block (the Llama-2 FFN
+ * the paper's models are built on, Sec. 4.1) whose hidden width h_i differs
+ * from expert to expert (Sec. 3.1).  Experts outside the top-k have gate
+ * softmax(-inf) = 0 and are never evaluated; every token is served by exactly
+ * k experts (no capacity limit, no dropped tokens).
+ *
+ * Notation: T tokens, d = d_model, N experts, k = top_k, h[e] = hidden width of
+ * expert e, S = sum_e h[e], off[e] = sum_{e'<e} h[e'].
+ *
+ * All pointers named "device" are CUDA device pointers owned by the caller.
+ * The library allocates no device memory; every call only enqueues kernels on
+ * the given stream and returns without synchronising.  No exception crosses
+ * this boundary and no call aborts: errors are returned as modse_status_t.
+ */
+#ifndef MODSE_H
+#define MODSE_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct modse_layer modse_layer_t; /* opaque host object owned by the library */
+
+typedef enum {
+    MODSE_OK = 0,
+    MODSE_ERR_INVALID_ARG = 1,         /* NULL/misaligned pointer, size out of range            */
+    MODSE_ERR_UNSUPPORTED = 2,         /* legal layer the CUDA path cannot run (see modse_create) */
+    MODSE_ERR_WORKSPACE_TOO_SMALL = 3, /* workspace_bytes < modse_workspace_bytes(...)           */
+    MODSE_ERR_STATE = 4,               /* backward without a matching saved forward              */
+    MODSE_ERR_CUDA = 5,                /* a CUDA runtime/driver call or launch failed            */
+    MODSE_ERR_DEVICE_TIMEOUT = 6,      /* a bounded wait inside a kernel expired                 */
+    MODSE_ERR_DEVICE_BOUNDS = 7        /* a kernel met an index outside its buffers              */
+} modse_status_t;
+
+typedef enum {
+    MODSE_F32 = 0, /* fp32 storage, fp32 FMA arithmetic                                   */
+    MODSE_BF16 = 1 /* bf16 storage, tensor-core products with fp32 accumulation           */
+} modse_dtype_t;
+
+/* ---- layer object ------------------------------------------------------- */
+
+/* Describes a layer (Sec. 3.1): d_model, N experts with hidden widths
+ * ffn_sizes[0..N) (copied), and k.  Host only; touches no GPU.
+ * Requirements: d_model >= 8 and a multiple of 8; 1 <= n_experts <= 256;
+ * 1 <= top_k <= n_experts; every width >= 16 and a multiple of 16.
+ * top_k > 2 is a legal layer the CUDA path does not run (MODSE_ERR_UNSUPPORTED).
+ * The bf16 type further needs d_model % 128 == 0 and every width % 64 == 0
+ * (checked by forward/backward, MODSE_ERR_UNSUPPORTED).
+ * The pair rule of Eq. 5-6 is not enforced (query it with modse_check_pairs).
+ * Returns NULL on error; modse_last_create_error() says why.                 */
+modse_layer_t *modse_create(int d_model, int n_experts, const int *ffn_sizes, int top_k);
+modse_status_t modse_last_create_error(void); /* per calling thread */
+modse_status_t modse_destroy(modse_layer_t *layer); /* NULL is accepted */
+
+/* Sec. 3.1, Eq. 5-6: returns 1 iff n_experts is even and every adjacent pair
+ * (2p, 2p+1) - "expert 0 and expert 1 on the same GPU, and so forth",
+ * Sec. 3.2 - has the same width sum 2h; *pair_sum_out (may be NULL) gets it.  */
+int modse_check_pairs(const int *ffn_sizes, int n_experts, int *pair_sum_out);
+
+const char *modse_status_string(modse_status_t status);
+
+/* ---- tensors ------------------------------------------------------------ */
+
+/* Weights, all row-major in the layer dtype, 16-byte aligned device pointers:
+ *   w_router [N, d]   row i gives logit i of H(x) = x . W_g             (Eq. 2)
+ *   w_gate   [S, d]   rows off[e] .. off[e]+h[e]-1 belong to expert e
+ *   w_up     [S, d]   same
+ *   w_down   [d, S]   columns off[e] .. off[e]+h[e]-1 belong to expert e
+ * Expert e computes  E_e(x) = W_down_e (silu(W_gate_e x) * (W_up_e x)).      */
+typedef struct {
+    const void *w_router;
+    const void *w_gate;
+    const void *w_up;
+    const void *w_down;
+} modse_weights_t;
+
+/* Weight gradients, same shapes and layouts; dw_router is always fp32, the
+ * others are in the layer dtype.  Overwritten (not accumulated) by backward;
+ * rows/columns of an expert that received no token are written as zeros.    */
+typedef struct {
+    void *dw_router;
+    void *dw_gate;
+    void *dw_up;
+    void *dw_down;
+} modse_wgrads_t;
+
+/* ---- calls -------------------------------------------------------------- */
+
+/* Bytes of device scratch a forward (and its backward, if save_for_backward)
+ * needs for n_tokens tokens.  0 on bad arguments.  The buffer must be 256-byte
+ * aligned and is owned by the caller; its content after forward holds the
+ * routing tables and, if saved, the activations backward consumes.           */
+size_t modse_workspace_bytes(const modse_layer_t *layer, modse_dtype_t dtype, int n_tokens,
+                             int save_for_backward);
+
+/* Eq. 2-4.  x [T, d] and y [T, d] device, layer dtype, row-major.
+ * Steps, all on `cuda_stream` (a cudaStream_t, NULL = legacy default stream):
+ * router logits + top-k + gates, per-expert counts/offsets and the stable
+ * permutation (expert groups ascending, tokens ascending inside a group),
+ * gather into expert groups, grouped up/gate projection with SwiGLU, grouped
+ * down projection, gate-weighted sum back in token order (slot 0 then slot 1).
+ * n_tokens == 0 is MODSE_OK and does nothing.                                */
+modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
+                             const void *x, int n_tokens, void *y, void *workspace,
+                             size_t workspace_bytes, int save_for_backward, void *cuda_stream);
+
+/* Exact gradient of modse_forward with the top-k selection held fixed (the
+ * selection is piecewise constant in x).  Needs the workspace of a preceding
+ * modse_forward(..., save_for_backward=1) on the same layer object, dtype and
+ * n_tokens (else MODSE_ERR_STATE) and the same x and weights.  dy [T, d] is
+ * the upstream gradient, dx [T, d] the result (layer dtype).  Gate and router
+ * gradients are computed and kept in fp32.  May be called repeatedly on one
+ * saved forward.                                                             */
+modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
+                              const void *x, const void *dy, int n_tokens, void *dx,
+                              const modse_wgrads_t *wgrads, void *workspace, size_t workspace_bytes,
+                              void *cuda_stream);
+
+/* Device pointers to the routing tables inside `workspace`, valid after a
+ * forward with the same layer/n_tokens until the workspace is reused.  Any
+ * output pointer may be NULL.  (Per-slot counts are what the paper's Appendix A
+ * tables list as "top0"/"top1".)
+ *   topk_idx [T,k] int32 (slot 0 = largest logit; ties go to the lower index)
+ *   topk_gate [T,k] fp32, counts [N], counts_slot [k,N], offsets [N+1],
+ *   row_of [T,k] (row of assignment (t,j) in expert-grouped order),
+ *   token_of [k*T] (inverse map)                                             */
+modse_status_t modse_get_routing(const modse_layer_t *layer, const void *workspace, int n_tokens,
+                                 const int **topk_idx, const float **topk_gate, const int **counts,
+                                 const int **counts_slot, const int **offsets, const int **row_of,
+                                 const int **token_of);
+
+/* Device pointers to the fp32 gate gradients dg [T,k] and logit gradients of
+ * the kept logits dz [T,k] written by modse_backward.                        */
+modse_status_t modse_get_gate_grads(const modse_layer_t *layer, const void *workspace, int n_tokens,
+                                    const float **dg, const float **dz);
+
+/* Synchronises the stream and reads the status word kernels write when a
+ * bounded wait expires or an index check fails; MODSE_OK if none did.        */
+modse_status_t modse_check_device_status(modse_layer_t *layer, const void *workspace, void *cuda_stream);
+
+/* Number of kernel launches the last forward/backward call on this layer
+ * enqueued (for launch accounting in benchmarks).                            */
+int modse_last_launch_count(const modse_layer_t *layer);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MODSE_H */
