@@ -1,0 +1,373 @@
+// Host side of libmodse: argument checking, workspace carving and the order in
+// which the stages of the MoDSE layer are enqueued (see include/modse.h).
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "modse_internal.h"
+#include "tc_gemm.h"
+
+struct modse_layer {
+    modse::LayerMeta meta;
+    std::vector<int> h;           // hidden widths
+    std::vector<int> h_desc;      // hidden widths, descending
+    // record of the last forward, checked by backward
+    const void *fwd_ws = nullptr;
+    int fwd_tokens = -1;
+    int fwd_dtype = -1;
+    int fwd_saved = 0;
+    int last_launches = 0;
+    modse::TcPlan tc;             // tensor-map cache of the bf16 path
+};
+
+namespace modse {
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool save)
+{
+    WsLayout L{};
+    L.T = T;
+    L.R = m.k * T;
+    L.Pmax = (int)align_up((size_t)L.R + (size_t)(kRowPad - 1) * m.N, kRowPad);
+    L.nblk = (T + kRouterTokB - 1) / kRouterTokB;
+    L.nblk_bwd = (T + kRouterBwdTokB - 1) / kRouterBwdTokB;
+    // sum_e cp_e*h_e <= T * (k largest widths) + (pad-1) * S
+    size_t topk_sum = 0;
+    for (int j = 0; j < m.k; ++j) topk_sum += (size_t)h_desc[j];
+    L.hb = (size_t)T * topk_sum + (size_t)(kRowPad - 1) * m.S;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    const size_t kT = (size_t)m.k * T, N = m.N;
+    L.status = take(64);
+    L.topk_idx = take(kT * 4);
+    L.topk_gate = take(kT * 4);
+    L.counts = take(N * 4);
+    L.counts_slot = take((size_t)m.k * N * 4);
+    L.offsets = take((N + 1) * 4);
+    L.poffsets = take((N + 1) * 4);
+    L.ebase = take((N + 1) * 8);
+    L.row_of = take(kT * 4);
+    L.token_of = take(kT * 4);
+    L.prow_of = take(kT * 4);
+    L.ptoken_of = take((size_t)L.Pmax * 4);
+    L.pgate = take((size_t)L.Pmax * 4);
+    L.block_counts = take((size_t)L.nblk * m.k * N * 4);
+    L.xp = take((size_t)L.Pmax * m.d * esz);
+    L.hm = take(L.hb * esz);
+    L.o = take((size_t)L.Pmax * m.d * esz);
+    if (save) {
+        L.a_pre = take(L.hb * esz);
+        L.b_pre = take(L.hb * esz);
+        L.dg = take(kT * 4);
+        L.dz = take(kT * 4);
+        L.dwr_partial = take((size_t)L.nblk_bwd * N * m.d * 4);
+        L.dyp = take((size_t)L.Pmax * m.d * esz);
+        L.da = take(L.hb * esz);
+        L.db = take(L.hb * esz);
+        L.dxp = take((size_t)L.Pmax * m.d * esz);
+    } else if (esz == 4) {
+        // the fp32 path always materialises the two pre-activations
+        L.a_pre = take(L.hb * esz);
+        L.b_pre = take(L.hb * esz);
+    }
+    L.total = off;
+    return L;
+}
+
+WsPtrs carve(void *ws, const WsLayout &L)
+{
+    unsigned char *b = static_cast<unsigned char *>(ws);
+    WsPtrs p{};
+    p.status = (int *)(b + L.status);
+    p.topk_idx = (int *)(b + L.topk_idx);
+    p.topk_gate = (float *)(b + L.topk_gate);
+    p.counts = (int *)(b + L.counts);
+    p.counts_slot = (int *)(b + L.counts_slot);
+    p.offsets = (int *)(b + L.offsets);
+    p.poffsets = (int *)(b + L.poffsets);
+    p.ebase = (long long *)(b + L.ebase);
+    p.row_of = (int *)(b + L.row_of);
+    p.token_of = (int *)(b + L.token_of);
+    p.prow_of = (int *)(b + L.prow_of);
+    p.ptoken_of = (int *)(b + L.ptoken_of);
+    p.pgate = (float *)(b + L.pgate);
+    p.block_counts = (int *)(b + L.block_counts);
+    p.dg = (float *)(b + L.dg);
+    p.dz = (float *)(b + L.dz);
+    p.dwr_partial = (float *)(b + L.dwr_partial);
+    p.xp = b + L.xp;
+    p.a_pre = b + L.a_pre;
+    p.b_pre = b + L.b_pre;
+    p.hm = b + L.hm;
+    p.o = b + L.o;
+    p.dyp = b + L.dyp;
+    p.da = b + L.da;
+    p.db = b + L.db;
+    p.dxp = b + L.dxp;
+    return p;
+}
+
+static thread_local modse_status_t g_create_error = MODSE_OK;
+
+static bool aligned16(const void *p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+// The bf16 tensor-core kernels tile the hidden axis in panels of 64 and the
+// model axis in tiles of 128.
+static bool tc_supported(const modse_layer *L)
+{
+    if (L->meta.d % 128 != 0) return false;
+    for (int h : L->h)
+        if (h % kPanel != 0) return false;
+    return true;
+}
+
+}  // namespace modse
+
+using namespace modse;
+
+extern "C" {
+
+modse_layer_t *modse_create(int d_model, int n_experts, const int *ffn_sizes, int top_k)
+{
+    g_create_error = MODSE_OK;
+    if (ffn_sizes == nullptr || d_model < 8 || d_model % 8 != 0 || n_experts < 1 || n_experts > kMaxExperts ||
+        top_k < 1 || top_k > n_experts) {
+        g_create_error = MODSE_ERR_INVALID_ARG;
+        return nullptr;
+    }
+    long long S = 0;
+    for (int e = 0; e < n_experts; ++e) {
+        if (ffn_sizes[e] < 16 || ffn_sizes[e] % 16 != 0) {
+            g_create_error = MODSE_ERR_INVALID_ARG;
+            return nullptr;
+        }
+        S += ffn_sizes[e];
+    }
+    if (S > (1ll << 30)) {
+        g_create_error = MODSE_ERR_INVALID_ARG;
+        return nullptr;
+    }
+    if (top_k > 2) {
+        g_create_error = MODSE_ERR_UNSUPPORTED;
+        return nullptr;
+    }
+    modse_layer *L = new (std::nothrow) modse_layer();
+    if (L == nullptr) {
+        g_create_error = MODSE_ERR_INVALID_ARG;
+        return nullptr;
+    }
+    L->meta.d = d_model;
+    L->meta.N = n_experts;
+    L->meta.k = top_k;
+    L->meta.S = (int)S;
+    L->meta.hoff[0] = 0;
+    for (int e = 0; e < n_experts; ++e) L->meta.hoff[e + 1] = L->meta.hoff[e] + ffn_sizes[e];
+    for (int e = n_experts + 1; e <= kMaxExperts; ++e) L->meta.hoff[e] = L->meta.hoff[n_experts];
+    L->h.assign(ffn_sizes, ffn_sizes + n_experts);
+    L->h_desc = L->h;
+    std::sort(L->h_desc.begin(), L->h_desc.end(), [](int a, int b) { return a > b; });
+    return L;
+}
+
+modse_status_t modse_last_create_error(void) { return g_create_error; }
+
+modse_status_t modse_destroy(modse_layer_t *layer)
+{
+    delete layer;
+    return MODSE_OK;
+}
+
+int modse_check_pairs(const int *ffn_sizes, int n_experts, int *pair_sum_out)
+{
+    if (ffn_sizes == nullptr || n_experts < 2 || n_experts % 2 != 0) return 0;
+    const int sum = ffn_sizes[0] + ffn_sizes[1];
+    for (int p = 1; p < n_experts / 2; ++p)
+        if (ffn_sizes[2 * p] + ffn_sizes[2 * p + 1] != sum) return 0;
+    if (pair_sum_out) *pair_sum_out = sum;
+    return 1;
+}
+
+const char *modse_status_string(modse_status_t s)
+{
+    switch (s) {
+    case MODSE_OK: return "ok";
+    case MODSE_ERR_INVALID_ARG: return "invalid argument";
+    case MODSE_ERR_UNSUPPORTED: return "unsupported layer shape";
+    case MODSE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case MODSE_ERR_STATE: return "backward without a matching saved forward";
+    case MODSE_ERR_CUDA: return "CUDA error";
+    case MODSE_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case MODSE_ERR_DEVICE_BOUNDS: return "a kernel met an index outside its buffers";
+    }
+    return "unknown status";
+}
+
+size_t modse_workspace_bytes(const modse_layer_t *layer, modse_dtype_t dtype, int n_tokens, int save_for_backward)
+{
+    if (layer == nullptr || n_tokens < 0 || (dtype != MODSE_F32 && dtype != MODSE_BF16)) return 0;
+    if ((long long)n_tokens * layer->meta.k > (1ll << 30)) return 0;
+    const WsLayout L = make_layout(layer->meta, layer->h_desc.data(), dtype == MODSE_F32 ? 4 : 2, n_tokens,
+                                   save_for_backward != 0);
+    return L.total;
+}
+
+#define MODSE_CUDA(expr)                               \
+    do {                                               \
+        cudaError_t ce__ = (expr);                     \
+        if (ce__ != cudaSuccess) return MODSE_ERR_CUDA; \
+    } while (0)
+
+static modse_status_t check_common(const modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *w,
+                                   int n_tokens, const void *workspace, size_t workspace_bytes, int save)
+{
+    if (layer == nullptr || w == nullptr || n_tokens < 0) return MODSE_ERR_INVALID_ARG;
+    if (dtype != MODSE_F32 && dtype != MODSE_BF16) return MODSE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MODSE_OK;
+    if ((long long)n_tokens * layer->meta.k > (1ll << 30)) return MODSE_ERR_INVALID_ARG;
+    if (!aligned16(w->w_router) || !aligned16(w->w_gate) || !aligned16(w->w_up) || !aligned16(w->w_down))
+        return MODSE_ERR_INVALID_ARG;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255) != 0) return MODSE_ERR_INVALID_ARG;
+    if (dtype == MODSE_BF16 && !tc_supported(layer)) return MODSE_ERR_UNSUPPORTED;
+    if (workspace_bytes < modse_workspace_bytes(layer, dtype, n_tokens, save)) return MODSE_ERR_WORKSPACE_TOO_SMALL;
+    return MODSE_OK;
+}
+
+modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
+                             const void *x, int n_tokens, void *y, void *workspace, size_t workspace_bytes,
+                             int save_for_backward, void *cuda_stream)
+{
+    modse_status_t st = check_common(layer, dtype, weights, n_tokens, workspace, workspace_bytes, save_for_backward);
+    if (st != MODSE_OK) return st;
+    if (n_tokens == 0) return MODSE_OK;
+    if (!aligned16(x) || !aligned16(y)) return MODSE_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const LayerMeta &m = layer->meta;
+    const bool save = save_for_backward != 0;
+    const WsLayout L = make_layout(m, layer->h_desc.data(), dtype == MODSE_F32 ? 4 : 2, n_tokens, save);
+    const WsPtrs p = carve(workspace, L);
+    int launches = 0;
+    layer->fwd_ws = nullptr;
+
+    MODSE_CUDA(cudaMemsetAsync(p.status, 0, 64, s));
+    MODSE_CUDA(launch_router(dtype, m, x, weights->w_router, n_tokens, p, s, &launches));
+    MODSE_CUDA(launch_rank(m, n_tokens, L.Pmax, p, s, &launches));
+    MODSE_CUDA(launch_permute(dtype, m, x, n_tokens, p, s, &launches));
+    if (dtype == MODSE_F32 || tc_force_simt()) {
+        // the bf16 cross-check path materialises both pre-activations, which only a saved forward has room for
+        if (dtype == MODSE_BF16 && !save) return MODSE_ERR_UNSUPPORTED;
+        SimtGemmArgs a{p.xp, weights->w_gate, p.a_pre, 0};
+        MODSE_CUDA(launch_simt_gemm(dtype, kUpGate, m, L.Pmax, p, a, s, &launches));
+        a.wgt = weights->w_up; a.out = p.b_pre;
+        MODSE_CUDA(launch_simt_gemm(dtype, kUpGate, m, L.Pmax, p, a, s, &launches));
+        MODSE_CUDA(launch_swiglu_fwd(dtype, m, p, L.hb, s, &launches));
+        SimtGemmArgs b{p.hm, weights->w_down, p.o, 0};
+        MODSE_CUDA(launch_simt_gemm(dtype, kDown, m, L.Pmax, p, b, s, &launches));
+    } else {
+        st = tc_forward(layer->tc, m, L, p, weights, save, s, &launches);
+        if (st != MODSE_OK) return st;
+    }
+    MODSE_CUDA(launch_combine(dtype, m, n_tokens, p, y, s, &launches));
+
+    layer->fwd_ws = workspace;
+    layer->fwd_tokens = n_tokens;
+    layer->fwd_dtype = (int)dtype;
+    layer->fwd_saved = save ? 1 : 0;
+    layer->last_launches = launches;
+    return MODSE_OK;
+}
+
+modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
+                              const void *x, const void *dy, int n_tokens, void *dx, const modse_wgrads_t *wgrads,
+                              void *workspace, size_t workspace_bytes, void *cuda_stream)
+{
+    modse_status_t st = check_common(layer, dtype, weights, n_tokens, workspace, workspace_bytes, 1);
+    if (st != MODSE_OK) return st;
+    if (wgrads == nullptr) return MODSE_ERR_INVALID_ARG;
+    if (n_tokens == 0) return MODSE_OK;
+    if (!aligned16(x) || !aligned16(dy) || !aligned16(dx) || !aligned16(wgrads->dw_router) ||
+        !aligned16(wgrads->dw_gate) || !aligned16(wgrads->dw_up) || !aligned16(wgrads->dw_down))
+        return MODSE_ERR_INVALID_ARG;
+    if (layer->fwd_ws != workspace || layer->fwd_tokens != n_tokens || layer->fwd_dtype != (int)dtype ||
+        !layer->fwd_saved)
+        return MODSE_ERR_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const LayerMeta &m = layer->meta;
+    const WsLayout L = make_layout(m, layer->h_desc.data(), dtype == MODSE_F32 ? 4 : 2, n_tokens, true);
+    const WsPtrs p = carve(workspace, L);
+    int launches = 0;
+
+    MODSE_CUDA(launch_dg_permute(dtype, m, dy, n_tokens, p, s, &launches));
+    if (dtype == MODSE_F32 || tc_force_simt()) {
+        SimtGemmArgs a{p.dyp, weights->w_down, p.da, 0};                       // dHm into the dA buffer
+        MODSE_CUDA(launch_simt_gemm(dtype, kDownDgrad, m, L.Pmax, p, a, s, &launches));
+        MODSE_CUDA(launch_swiglu_bwd(dtype, m, p, L.hb, s, &launches));
+        SimtGemmArgs w{p.dyp, p.hm, wgrads->dw_down, 0};
+        MODSE_CUDA(launch_simt_gemm(dtype, kDownWgrad, m, L.Pmax, p, w, s, &launches));
+        SimtGemmArgs g{p.da, weights->w_gate, p.dxp, 0};
+        MODSE_CUDA(launch_simt_gemm(dtype, kUpGateDgrad, m, L.Pmax, p, g, s, &launches));
+        g.act = p.db; g.wgt = weights->w_up; g.accumulate = 1;
+        MODSE_CUDA(launch_simt_gemm(dtype, kUpGateDgrad, m, L.Pmax, p, g, s, &launches));
+        SimtGemmArgs wg{p.da, p.xp, wgrads->dw_gate, 0};
+        MODSE_CUDA(launch_simt_gemm(dtype, kUpGateWgrad, m, L.Pmax, p, wg, s, &launches));
+        wg.act = p.db; wg.out = wgrads->dw_up;
+        MODSE_CUDA(launch_simt_gemm(dtype, kUpGateWgrad, m, L.Pmax, p, wg, s, &launches));
+    } else {
+        st = tc_backward(layer->tc, m, L, p, weights, wgrads, s, &launches);
+        if (st != MODSE_OK) return st;
+    }
+    MODSE_CUDA(launch_router_bwd(dtype, m, x, weights->w_router, n_tokens, L.nblk_bwd, p, dx,
+                                 static_cast<float *>(wgrads->dw_router), s, &launches));
+    layer->last_launches = launches;
+    return MODSE_OK;
+}
+
+modse_status_t modse_get_routing(const modse_layer_t *layer, const void *workspace, int n_tokens,
+                                 const int **topk_idx, const float **topk_gate, const int **counts,
+                                 const int **counts_slot, const int **offsets, const int **row_of,
+                                 const int **token_of)
+{
+    if (layer == nullptr || workspace == nullptr || n_tokens < 1) return MODSE_ERR_INVALID_ARG;
+    if (layer->fwd_ws != workspace || layer->fwd_tokens != n_tokens) return MODSE_ERR_STATE;
+    const WsLayout L = make_layout(layer->meta, layer->h_desc.data(), layer->fwd_dtype == MODSE_F32 ? 4 : 2,
+                                   n_tokens, layer->fwd_saved != 0);
+    const WsPtrs p = carve(const_cast<void *>(workspace), L);
+    if (topk_idx) *topk_idx = p.topk_idx;
+    if (topk_gate) *topk_gate = p.topk_gate;
+    if (counts) *counts = p.counts;
+    if (counts_slot) *counts_slot = p.counts_slot;
+    if (offsets) *offsets = p.offsets;
+    if (row_of) *row_of = p.row_of;
+    if (token_of) *token_of = p.token_of;
+    return MODSE_OK;
+}
+
+modse_status_t modse_get_gate_grads(const modse_layer_t *layer, const void *workspace, int n_tokens,
+                                    const float **dg, const float **dz)
+{
+    if (layer == nullptr || workspace == nullptr || n_tokens < 1) return MODSE_ERR_INVALID_ARG;
+    if (layer->fwd_ws != workspace || layer->fwd_tokens != n_tokens || !layer->fwd_saved) return MODSE_ERR_STATE;
+    const WsLayout L = make_layout(layer->meta, layer->h_desc.data(), layer->fwd_dtype == MODSE_F32 ? 4 : 2,
+                                   n_tokens, true);
+    const WsPtrs p = carve(const_cast<void *>(workspace), L);
+    if (dg) *dg = p.dg;
+    if (dz) *dz = p.dz;
+    return MODSE_OK;
+}
+
+modse_status_t modse_check_device_status(modse_layer_t *layer, const void *workspace, void *cuda_stream)
+{
+    if (layer == nullptr || workspace == nullptr) return MODSE_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return MODSE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (word == kDevTimeout) return MODSE_ERR_DEVICE_TIMEOUT;
+    if (word == kDevBounds) return MODSE_ERR_DEVICE_BOUNDS;
+    return MODSE_OK;
+}
+
+int modse_last_launch_count(const modse_layer_t *layer) { return layer ? layer->last_launches : 0; }
+
+}  // extern "C"

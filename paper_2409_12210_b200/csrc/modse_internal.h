@@ -1,0 +1,90 @@
+// Internal declarations shared by the CUDA translation units of libmodse.
+// Nothing here is part of the public ABI (include/modse.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "modse.h"
+
+namespace modse {
+
+constexpr int kMaxExperts = 256;
+constexpr int kRowPad = 128;        // every expert group is padded to a multiple of this many rows
+constexpr int kRouterTokB = 64;     // tokens per block in the router / rank kernels
+constexpr int kRouterBwdTokB = 128; // tokens per block in the router backward kernel
+constexpr int kPanel = 64;          // hidden-axis panel width of the bf16 activation layout
+
+// Device status word values (first int of the workspace).
+enum : int { kDevOk = 0, kDevTimeout = 1, kDevBounds = 2 };
+
+// Layer shape, passed by value to kernels (prefix sums of the hidden widths).
+struct LayerMeta {
+    int d, N, k, S;
+    int hoff[kMaxExperts + 1];
+};
+
+// Byte offsets of every region inside the caller's workspace.
+struct WsLayout {
+    int T, R, Pmax, nblk, nblk_bwd;
+    size_t hb;   // element capacity of each [padded rows x h_e] activation buffer
+    size_t status, topk_idx, topk_gate, counts, counts_slot, offsets, poffsets, ebase, row_of, token_of,
+        prow_of, ptoken_of, pgate, block_counts, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
+        total;
+};
+
+// Pointers carved out of the workspace (device addresses).
+struct WsPtrs {
+    int *status, *topk_idx;
+    float *topk_gate;
+    int *counts, *counts_slot, *offsets, *poffsets;
+    long long *ebase;
+    int *row_of, *token_of, *prow_of, *ptoken_of;
+    float *pgate;
+    int *block_counts;
+    float *dg, *dz, *dwr_partial;
+    void *xp, *a_pre, *b_pre, *hm, *o, *dyp, *da, *db, *dxp;
+};
+
+WsLayout make_layout(const LayerMeta &m, const int *h_sorted_desc, int elem_bytes, int T, bool save);
+WsPtrs carve(void *ws, const WsLayout &L);
+
+// ---- routing / permutation / elementwise stages (routing_kernels.cu) ----
+cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
+                          const WsPtrs &p, cudaStream_t s, int *launches);
+cudaError_t launch_rank(const LayerMeta &m, int T, int Pmax, const WsPtrs &p, cudaStream_t s, int *launches);
+cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, const WsPtrs &p,
+                           cudaStream_t s, int *launches);
+cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, cudaStream_t s,
+                           int *launches);
+cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, const WsPtrs &p,
+                              cudaStream_t s, int *launches);
+cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
+                              int nblk_bwd, const WsPtrs &p, void *dx, float *dw_router, cudaStream_t s,
+                              int *launches);
+
+// ---- fp32-FMA grouped GEMMs and SwiGLU elementwise (simt_gemm.cu) ----
+enum GemmKind : int {
+    kUpGate = 0,      // C[cp_e, h_e]  = xp_e  . W_e^T          (W = w_gate or w_up)
+    kDown = 1,        // o[cp_e, d]    = Hm_e  . W_down_e^T
+    kDownDgrad = 2,   // dHm[cp_e,h_e] = dyp_e . W_down_e
+    kDownWgrad = 3,   // dW_down_e[d,h_e] = dyp_e^T . Hm_e
+    kUpGateDgrad = 4, // dxp[cp_e, d] (+)= dA_e . W_e
+    kUpGateWgrad = 5  // dW_e[h_e, d]  = dA_e^T . xp_e
+};
+struct SimtGemmArgs {
+    const void *act;   // activation operand in padded expert-grouped rows ([P,d]) or [rows,h_e] buffer
+    const void *wgt;   // weight operand, or second activation operand for the weight-gradient kinds
+    void *out;
+    int accumulate;    // 1: out += product
+};
+cudaError_t launch_simt_gemm(modse_dtype_t dt, GemmKind kind, const LayerMeta &m, int Pmax, const WsPtrs &p,
+                             const SimtGemmArgs &a, cudaStream_t s, int *launches);
+cudaError_t launch_swiglu_fwd(modse_dtype_t dt, const LayerMeta &m, const WsPtrs &p, size_t hb, cudaStream_t s,
+                              int *launches);
+cudaError_t launch_swiglu_bwd(modse_dtype_t dt, const LayerMeta &m, const WsPtrs &p, size_t hb, cudaStream_t s,
+                              int *launches);
+
+}  // namespace modse

@@ -1,0 +1,599 @@
+// Router, permutation bookkeeping and the memory-bound stages around the
+// grouped GEMMs of the MoDSE layer.
+//
+//   router_kernel      H(x) = x . W_g, top-k with ties to the lower index,
+//                      softmax over the kept logits (Sec. 2, Eq. 2-3), and a
+//                      per-block, per-slot histogram of the chosen experts.
+//   rank_kernel        exclusive scans of the histogram -> counts, offsets and
+//                      the stable destination row of every (token, slot).
+//   permute_kernel     gathers token rows into padded expert groups.
+//   combine_kernel     y_t = sum_j g[t,j] * o[row(t,j)]  (Sec. 3.1, Eq. 4).
+//   dg_permute_kernel  dg[t,j] = <dY_t, o_(t,j)>, rows g*dY_t in group order.
+//   router_bwd_kernel  softmax Jacobian on the kept logits, dx assembly and
+//                      per-block partial sums of dW_router; reduced in block
+//                      order by reduce_dwr_kernel so the result is reproducible.
+//
+// No kernel uses a floating-point atomic; every sum has a fixed order.
+#include "modse_internal.h"
+
+namespace modse {
+
+namespace {
+
+__device__ __forceinline__ void load8(const float *p, float (&v)[8])
+{
+    float4 a = *reinterpret_cast<const float4 *>(p);
+    float4 b = *reinterpret_cast<const float4 *>(p + 4);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&v)[8])
+{
+    uint4 q = *reinterpret_cast<const uint4 *>(p);
+    const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+}
+
+__device__ __forceinline__ void store8(float *p, const float (&v)[8])
+{
+    *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4 *>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
+}
+
+__device__ __forceinline__ void store8(__nv_bfloat16 *p, const float (&v)[8])
+{
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+        w[i] = *reinterpret_cast<uint32_t *>(&t);
+    }
+    *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+constexpr int kNoIndex = 0x7FFFFFFF;
+
+// ---------------------------------------------------------------------------
+// Router: one warp per token.  Each lane accumulates its 8-element chunks of
+// the row in ascending order with fp32 FMAs, then a butterfly adds the lanes.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok, int d, int N, int k,
+              int *__restrict__ topk_idx, float *__restrict__ topk_gate, int *__restrict__ block_counts,
+              int w_in_smem)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int Npad = (N + 3) & ~3;
+    int *cnt = reinterpret_cast<int *>(smem_raw);                                          // [k*N]
+    float *zbuf = reinterpret_cast<float *>(smem_raw + sizeof(int) * ((k * N + 3) & ~3));  // [8][Npad]
+    T *wsm = reinterpret_cast<T *>(reinterpret_cast<unsigned char *>(zbuf) + sizeof(float) * 8 * Npad);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int i = tid; i < k * N; i += blockDim.x) cnt[i] = 0;
+    const T *w = w_router;
+    if (w_in_smem) {
+        const size_t bytes = (size_t)N * d * sizeof(T);   // a multiple of 16: d is a multiple of 8
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(w_router);
+        unsigned char *dst = reinterpret_cast<unsigned char *>(wsm);
+        for (size_t i = (size_t)tid * 16; i < bytes; i += (size_t)blockDim.x * 16)
+            *reinterpret_cast<uint4 *>(dst + i) = *reinterpret_cast<const uint4 *>(src + i);
+        w = wsm;
+    }
+    __syncthreads();
+
+    float *z = zbuf + warp * Npad;
+    const int t0 = blockIdx.x * kRouterTokB;
+    for (int tok = warp; tok < kRouterTokB; tok += 8) {
+        const int t = t0 + tok;
+        if (t >= Ttok) break;
+        const T *xr = x + (size_t)t * d;
+        for (int g0 = 0; g0 < N; g0 += 8) {
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            for (int c = lane * 8; c < d; c += 256) {
+                float xv[8];
+                load8(xr + c, xv);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (g0 + i < N) {
+                        float wv[8];
+                        load8(w + (size_t)(g0 + i) * d + c, wv);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) acc[i] = fmaf(xv[u], wv[u], acc[i]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                float s = warp_sum(acc[i]);
+                if (lane == 0 && g0 + i < N) z[g0 + i] = s;
+            }
+        }
+        __syncwarp();
+        // KeepTopK: k rounds of arg-max over the logits not yet taken; the pair
+        // (value, index) is ordered so that equal values prefer the lower index.
+        float zsel[2] = {0.f, 0.f};
+        int isel[2] = {kNoIndex, kNoIndex};
+        for (int j = 0; j < k; ++j) {
+            float bv = -INFINITY;
+            int bi = kNoIndex;
+            for (int i = lane; i < N; i += 32) {
+                const bool taken = (j > 0 && i == isel[0]);
+                const float v = z[i];
+                if (!taken && (bi == kNoIndex || v > bv)) { bv = v; bi = i; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+                const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+                if (oi != kNoIndex && (bi == kNoIndex || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
+            }
+            zsel[j] = bv;
+            isel[j] = bi;
+        }
+        if (lane == 0) {
+            // Softmax over the kept logits (the others are -inf and contribute 0).
+            if (k == 1) {
+                topk_idx[t] = isel[0];
+                topk_gate[t] = 1.0f;
+                atomicAdd(&cnt[isel[0]], 1);
+            } else {
+                const float w1 = expf(zsel[1] - zsel[0]);
+                const float den = 1.0f + w1;
+                topk_idx[2 * (size_t)t] = isel[0];
+                topk_idx[2 * (size_t)t + 1] = isel[1];
+                topk_gate[2 * (size_t)t] = 1.0f / den;
+                topk_gate[2 * (size_t)t + 1] = w1 / den;
+                atomicAdd(&cnt[isel[0]], 1);
+                atomicAdd(&cnt[N + isel[1]], 1);
+            }
+        }
+        __syncwarp();
+    }
+    __syncthreads();
+    for (int i = tid; i < k * N; i += blockDim.x) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
+}
+
+// ---------------------------------------------------------------------------
+// Rank: block b owns tokens [b*64, b*64+64).  It sums the histograms of the
+// blocks before it (tokens before its own), scans the totals over experts, and
+// ranks its own assignments by token index.  Integer work only.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+rank_kernel(LayerMeta m, int Ttok, int Pmax, int nblk, const int *__restrict__ block_counts,
+            const int *__restrict__ topk_idx, const float *__restrict__ topk_gate, int *__restrict__ counts,
+            int *__restrict__ counts_slot, int *__restrict__ offsets, int *__restrict__ poffsets,
+            long long *__restrict__ ebase, int *__restrict__ row_of, int *__restrict__ token_of,
+            int *__restrict__ prow_of, int *__restrict__ ptoken_of, float *__restrict__ pgate, int *status)
+{
+    const int N = m.N, k = m.k, kN = k * N;
+    extern __shared__ int sm[];
+    int *tot = sm;                 // [kN] totals per (slot, expert)
+    int *pre = tot + kN;           // [kN] sum over earlier blocks
+    int *off = pre + kN;           // [N+1]
+    int *poff = off + N + 1;       // [N+1]
+    int *base = poff + N + 1;      // [N] rows of expert e taken by earlier blocks
+    int *bidx = base + N;          // [64*k] this block's expert choices
+
+    const int tid = threadIdx.x, b = blockIdx.x;
+    for (int p = tid; p < kN; p += 256) {
+        int before = 0, all = 0;
+        for (int bb = 0; bb < nblk; ++bb) {
+            const int c = block_counts[(size_t)bb * kN + p];
+            all += c;
+            if (bb < b) before += c;
+        }
+        tot[p] = all;
+        pre[p] = before;
+    }
+    const int t0 = b * kRouterTokB;
+    for (int i = tid; i < kRouterTokB * k; i += 256) {
+        const int t = t0 + i / k;
+        bidx[i] = (t < Ttok) ? topk_idx[(size_t)t0 * k + i] : -1;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int o = 0, po = 0;
+        long long eb = 0;
+        for (int e = 0; e < N; ++e) {
+            int c = 0, bs = 0;
+            for (int j = 0; j < k; ++j) { c += tot[j * N + e]; bs += pre[j * N + e]; }
+            off[e] = o;
+            poff[e] = po;
+            base[e] = bs;
+            if (b == 0) {
+                counts[e] = c;
+                offsets[e] = o;
+                poffsets[e] = po;
+                ebase[e] = eb;
+            }
+            const int cp = (c + kRowPad - 1) / kRowPad * kRowPad;
+            eb += (long long)cp * (m.hoff[e + 1] - m.hoff[e]);
+            o += c;
+            po += cp;
+        }
+        off[N] = o;
+        poff[N] = po;
+        if (b == 0) {
+            offsets[N] = o;
+            poffsets[N] = po;
+            ebase[N] = eb;
+            if (po > Pmax || o != k * Ttok) atomicMax(status, kDevBounds);
+        }
+    }
+    __syncthreads();
+    if (b == 0)
+        for (int i = tid; i < kN; i += 256) counts_slot[i] = tot[i];
+
+    // Rank inside the block: assignments of the same expert from earlier tokens.
+    for (int i = tid; i < kRouterTokB * k; i += 256) {
+        const int e = bidx[i];
+        if (e < 0 || e >= N) continue;
+        const int tl = i / k;
+        int r = 0;
+        for (int q = 0; q < tl * k; ++q) r += (bidx[q] == e);
+        const int t = t0 + tl;
+        const int local = base[e] + r;
+        const int row = off[e] + local, prow = poff[e] + local;
+        row_of[(size_t)t * k + (i % k)] = row;
+        prow_of[(size_t)t * k + (i % k)] = prow;
+        if (row < k * Ttok) token_of[row] = t;
+        if (prow < Pmax) {
+            ptoken_of[prow] = t;
+            pgate[prow] = topk_gate[(size_t)t * k + (i % k)];
+        }
+    }
+    // Padding rows of every group (and the unused tail) carry token -1, gate 0.
+    if (b == 0) {
+        for (int e = 0; e < N; ++e) {
+            const int c = off[e + 1] - off[e];
+            for (int r = poff[e] + c + tid; r < poff[e + 1] && r < Pmax; r += 256) { ptoken_of[r] = -1; pgate[r] = 0.f; }
+        }
+        for (int r = poff[N] + tid; r < Pmax; r += 256) { ptoken_of[r] = -1; pgate[r] = 0.f; }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Permute: one warp per token reads the row once and writes it to the k rows
+// it owns in the padded expert-grouped buffer.  Extra blocks zero the padding.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int *__restrict__ prow_of,
+               const int *__restrict__ counts, const int *__restrict__ poffsets, T *__restrict__ xp, int tok_blocks)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if ((int)blockIdx.x < tok_blocks) {
+        const int t = blockIdx.x * 8 + warp;
+        if (t >= Ttok) return;
+        const T *src = x + (size_t)t * d;
+        int rows[2];
+        rows[0] = prow_of[(size_t)t * k];
+        rows[1] = (k > 1) ? prow_of[(size_t)t * k + 1] : -1;
+        for (int c = lane * 8; c < d; c += 256) {
+            float v[8];
+            load8(src + c, v);
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+                if (rows[j] >= 0) store8(xp + (size_t)rows[j] * d + c, v);
+        }
+    } else {
+        // padding rows: 16 blocks of 8 warps per expert cover its (at most 127) pad rows
+        const int pb = blockIdx.x - tok_blocks;
+        const int e = pb / 16, i = (pb % 16) * 8 + warp;
+        if (e >= N) return;
+        const int row = poffsets[e] + counts[e] + i;
+        if (row >= poffsets[e + 1]) return;
+        const float zero[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int c = lane * 8; c < d; c += 256) store8(xp + (size_t)row * d + c, zero);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Combine (Eq. 4): y_t = g[t,0]*o[row(t,0)] + g[t,1]*o[row(t,1)], fp32, slot order.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+combine_kernel(const T *__restrict__ o, int Ttok, int d, int k, const int *__restrict__ prow_of,
+               const float *__restrict__ topk_gate, T *__restrict__ y)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * 8 + warp;
+    if (t >= Ttok) return;
+    const int r0 = prow_of[(size_t)t * k];
+    const float g0 = topk_gate[(size_t)t * k];
+    const int r1 = (k > 1) ? prow_of[(size_t)t * k + 1] : -1;
+    const float g1 = (k > 1) ? topk_gate[(size_t)t * k + 1] : 0.f;
+    for (int c = lane * 8; c < d; c += 256) {
+        float a[8], acc[8];
+        load8(o + (size_t)r0 * d + c, a);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc[u] = g0 * a[u];
+        if (r1 >= 0) {
+            load8(o + (size_t)r1 * d + c, a);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) acc[u] = fmaf(g1, a[u], acc[u]);
+        }
+        store8(y + (size_t)t * d + c, acc);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Backward entry: dg[t,j] = <dY_t, o_(t,j)>; dyp[row(t,j)] = g[t,j]*dY_t.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+dg_permute_kernel(const T *__restrict__ dy, const T *__restrict__ o, int Ttok, int d, int N, int k,
+                  const int *__restrict__ prow_of, const float *__restrict__ topk_gate,
+                  const int *__restrict__ counts, const int *__restrict__ poffsets, float *__restrict__ dg,
+                  T *__restrict__ dyp, int tok_blocks)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if ((int)blockIdx.x < tok_blocks) {
+        const int t = blockIdx.x * 8 + warp;
+        if (t >= Ttok) return;
+        const T *src = dy + (size_t)t * d;
+        for (int j = 0; j < k; ++j) {
+            const int row = prow_of[(size_t)t * k + j];
+            const float g = topk_gate[(size_t)t * k + j];
+            float acc = 0.f;
+            for (int c = lane * 8; c < d; c += 256) {
+                float v[8], ov[8], sv[8];
+                load8(src + c, v);
+                load8(o + (size_t)row * d + c, ov);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { acc = fmaf(v[u], ov[u], acc); sv[u] = g * v[u]; }
+                store8(dyp + (size_t)row * d + c, sv);
+            }
+            acc = warp_sum(acc);
+            if (lane == 0) dg[(size_t)t * k + j] = acc;
+        }
+    } else {
+        const int pb = blockIdx.x - tok_blocks;
+        const int e = pb / 16, i = (pb % 16) * 8 + warp;
+        if (e >= N) return;
+        const int row = poffsets[e] + counts[e] + i;
+        if (row >= poffsets[e + 1]) return;
+        const float zero[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int c = lane * 8; c < d; c += 256) store8(dyp + (size_t)row * d + c, zero);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Router backward.  Phase A (warp per token): s = sum_j g_j dg_j,
+// dz_j = g_j (dg_j - s), dx_t = sum_j dxp[row_j] + sum_j dz_j W_router[e_j].
+// Phase B (thread per column): partial dW_router over this block's tokens in
+// ascending token order, kept in shared memory [N][dc] and written out.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+router_bwd_kernel(const T *__restrict__ x, const T *__restrict__ w_router, const T *__restrict__ dxp, int Ttok,
+                  int d, int N, int k, int dc, const int *__restrict__ topk_idx,
+                  const float *__restrict__ topk_gate, const int *__restrict__ prow_of,
+                  const float *__restrict__ dg, float *__restrict__ dz, T *__restrict__ dx,
+                  float *__restrict__ dwr_partial)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *dzs = reinterpret_cast<float *>(smem_raw);                    // [128][2]
+    int *idxs = reinterpret_cast<int *>(dzs + kRouterBwdTokB * 2);       // [128][2]
+    float *acc = reinterpret_cast<float *>(idxs + kRouterBwdTokB * 2);   // [N][dc]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t0 = blockIdx.x * kRouterBwdTokB;
+    const int c0 = blockIdx.y * dc;
+    const int cw = min(dc, d - c0);
+
+    for (int tl = warp; tl < kRouterBwdTokB; tl += 8) {
+        const int t = t0 + tl;
+        if (t >= Ttok) {
+            if (lane < 2) { dzs[tl * 2 + lane] = 0.f; idxs[tl * 2 + lane] = 0; }
+            continue;
+        }
+        float g[2] = {0.f, 0.f}, dgv[2] = {0.f, 0.f}, dzv[2];
+        int e[2] = {0, 0}, rows[2] = {-1, -1};
+        for (int j = 0; j < k; ++j) {
+            g[j] = topk_gate[(size_t)t * k + j];
+            dgv[j] = dg[(size_t)t * k + j];
+            e[j] = topk_idx[(size_t)t * k + j];
+            rows[j] = prow_of[(size_t)t * k + j];
+        }
+        const float s = g[0] * dgv[0] + g[1] * dgv[1];
+        dzv[0] = g[0] * (dgv[0] - s);
+        dzv[1] = g[1] * (dgv[1] - s);
+        if (lane < 2) {
+            dzs[tl * 2 + lane] = (lane < k) ? dzv[lane] : 0.f;
+            idxs[tl * 2 + lane] = e[lane];
+            if (blockIdx.y == 0 && lane < k) dz[(size_t)t * k + lane] = dzv[lane];
+        }
+        if (blockIdx.y == 0) {
+            for (int c = lane * 8; c < d; c += 256) {
+                float a[8], out[8], wv[8];
+                load8(dxp + (size_t)rows[0] * d + c, out);
+                if (k > 1) {
+                    load8(dxp + (size_t)rows[1] * d + c, a);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) out[u] += a[u];
+                }
+                for (int j = 0; j < k; ++j) {
+                    load8(w_router + (size_t)e[j] * d + c, wv);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) out[u] = fmaf(dzv[j], wv[u], out[u]);
+                }
+                store8(dx + (size_t)t * d + c, out);
+            }
+        }
+    }
+    for (int i = tid; i < N * dc; i += 256) acc[i] = 0.f;
+    __syncthreads();
+    const int ntok = min(kRouterBwdTokB, Ttok - t0);
+    for (int c = tid; c < cw; c += 256) {
+        for (int tl = 0; tl < ntok; ++tl) {
+            float xv;
+            if (sizeof(T) == 4) xv = reinterpret_cast<const float *>(x)[(size_t)(t0 + tl) * d + c0 + c];
+            else xv = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(x)[(size_t)(t0 + tl) * d + c0 + c]);
+            for (int j = 0; j < k; ++j) {
+                float *a = &acc[idxs[tl * 2 + j] * dc + c];
+                *a = fmaf(dzs[tl * 2 + j], xv, *a);
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < N * cw; i += 256) {
+        const int e = i / cw, c = i % cw;
+        dwr_partial[((size_t)blockIdx.x * N + e) * d + c0 + c] = acc[e * dc + c];
+    }
+}
+
+__global__ void __launch_bounds__(256)
+reduce_dwr_kernel(const float *__restrict__ partial, int nblk, int n, float *__restrict__ dwr)
+{
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= n) return;
+    float s = 0.f;
+    for (int b = 0; b < nblk; ++b) s += partial[(size_t)b * n + i];
+    dwr[i] = s;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------
+// Host launchers
+// ---------------------------------------------------------------------------
+#define MODSE_LAUNCH_CHECK()                        \
+    do {                                            \
+        cudaError_t e__ = cudaGetLastError();       \
+        if (e__ != cudaSuccess) return e__;         \
+        if (launches) ++*launches;                  \
+    } while (0)
+
+cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
+                          const WsPtrs &p, cudaStream_t s, int *launches)
+{
+    const int nblk = (T + kRouterTokB - 1) / kRouterTokB;
+    const size_t esz = dt == MODSE_F32 ? 4 : 2;
+    const size_t base = sizeof(int) * ((m.k * m.N + 3) & ~3) + sizeof(float) * 8 * ((m.N + 3) & ~3);
+    const size_t wbytes = (size_t)m.N * m.d * esz;
+    const int w_in_smem = (base + wbytes <= 160 * 1024) ? 1 : 0;
+    const size_t smem = base + (w_in_smem ? wbytes : 0);
+    if (dt == MODSE_F32) {
+        auto kern = router_kernel<float>;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<nblk, 256, smem, s>>>((const float *)x, (const float *)w_router, T, m.d, m.N, m.k, p.topk_idx,
+                                     p.topk_gate, p.block_counts, w_in_smem);
+    } else {
+        auto kern = router_kernel<__nv_bfloat16>;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<nblk, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
+                                     p.topk_idx, p.topk_gate, p.block_counts, w_in_smem);
+    }
+    MODSE_LAUNCH_CHECK();
+    return cudaSuccess;
+}
+
+cudaError_t launch_rank(const LayerMeta &m, int T, int Pmax, const WsPtrs &p, cudaStream_t s, int *launches)
+{
+    const int nblk = (T + kRouterTokB - 1) / kRouterTokB;
+    const int kN = m.k * m.N;
+    const size_t smem = sizeof(int) * (2 * kN + 2 * (m.N + 1) + m.N + kRouterTokB * m.k);
+    rank_kernel<<<nblk, 256, smem, s>>>(m, T, Pmax, nblk, p.block_counts, p.topk_idx, p.topk_gate, p.counts,
+                                        p.counts_slot, p.offsets, p.poffsets, p.ebase, p.row_of, p.token_of,
+                                        p.prow_of, p.ptoken_of, p.pgate, p.status);
+    MODSE_LAUNCH_CHECK();
+    return cudaSuccess;
+}
+
+cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, const WsPtrs &p,
+                           cudaStream_t s, int *launches)
+{
+    const int tok_blocks = (T + 7) / 8;
+    const int grid = tok_blocks + m.N * 16;
+    if (dt == MODSE_F32)
+        permute_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.prow_of, p.counts,
+                                                   p.poffsets, (float *)p.xp, tok_blocks);
+    else
+        permute_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k, p.prow_of,
+                                                           p.counts, p.poffsets, (__nv_bfloat16 *)p.xp, tok_blocks);
+    MODSE_LAUNCH_CHECK();
+    return cudaSuccess;
+}
+
+cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, cudaStream_t s,
+                           int *launches)
+{
+    const int grid = (T + 7) / 8;
+    if (dt == MODSE_F32)
+        combine_kernel<float><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of, p.topk_gate,
+                                                   (float *)y);
+    else
+        combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)p.o, T, m.d, m.k, p.prow_of,
+                                                           p.topk_gate, (__nv_bfloat16 *)y);
+    MODSE_LAUNCH_CHECK();
+    return cudaSuccess;
+}
+
+cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, const WsPtrs &p,
+                              cudaStream_t s, int *launches)
+{
+    const int tok_blocks = (T + 7) / 8;
+    const int grid = tok_blocks + m.N * 16;
+    if (dt == MODSE_F32)
+        dg_permute_kernel<float><<<grid, 256, 0, s>>>((const float *)dy, (const float *)p.o, T, m.d, m.N, m.k,
+                                                      p.prow_of, p.topk_gate, p.counts, p.poffsets, p.dg,
+                                                      (float *)p.dyp, tok_blocks);
+    else
+        dg_permute_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)dy,
+                                                              (const __nv_bfloat16 *)p.o, T, m.d, m.N, m.k,
+                                                              p.prow_of, p.topk_gate, p.counts, p.poffsets, p.dg,
+                                                              (__nv_bfloat16 *)p.dyp, tok_blocks);
+    MODSE_LAUNCH_CHECK();
+    return cudaSuccess;
+}
+
+cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
+                              int nblk_bwd, const WsPtrs &p, void *dx, float *dw_router, cudaStream_t s,
+                              int *launches)
+{
+    // column chunk so that the [N][dc] fp32 accumulator fits in 64 KB of shared memory
+    int dc = m.d;
+    while ((size_t)m.N * dc * 4 > 64 * 1024 && dc > 8) dc = (dc / 2 + 7) & ~7;
+    const int ychunks = (m.d + dc - 1) / dc;
+    const size_t smem =
+        sizeof(float) * kRouterBwdTokB * 2 + sizeof(int) * kRouterBwdTokB * 2 + sizeof(float) * m.N * dc;
+    dim3 grid(nblk_bwd, ychunks);
+    if (dt == MODSE_F32) {
+        auto kern = router_bwd_kernel<float>;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, 256, smem, s>>>((const float *)x, (const float *)w_router, (const float *)p.dxp, T, m.d, m.N,
+                                     m.k, dc, p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz, (float *)dx,
+                                     p.dwr_partial);
+    } else {
+        auto kern = router_bwd_kernel<__nv_bfloat16>;
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router,
+                                     (const __nv_bfloat16 *)p.dxp, T, m.d, m.N, m.k, dc, p.topk_idx, p.topk_gate,
+                                     p.prow_of, p.dg, p.dz, (__nv_bfloat16 *)dx, p.dwr_partial);
+    }
+    MODSE_LAUNCH_CHECK();
+    const int n = m.N * m.d;
+    reduce_dwr_kernel<<<(n + 255) / 256, 256, 0, s>>>(p.dwr_partial, nblk_bwd, n, dw_router);
+    MODSE_LAUNCH_CHECK();
+    return cudaSuccess;
+}
+
+}  // namespace modse
