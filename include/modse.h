@@ -151,6 +151,12 @@ modse_status_t modse_check_device_status(modse_layer_t *layer, const void *works
  * enqueued (for launch accounting in benchmarks).                            */
 int modse_last_launch_count(const modse_layer_t *layer);
 
+/* Debugging aid, process-wide: when on, bf16 layers run their grouped GEMMs on
+ * the fp32-FMA kernels of the fp32 type (with bf16 storage) instead of the
+ * tensor-core kernels - slow, meant for cross-checking.  Such a forward must
+ * be called with save_for_backward = 1.  Off by default.                    */
+void modse_debug_use_fma_path(int on);
+
 #ifdef __cplusplus
 }
 #endif

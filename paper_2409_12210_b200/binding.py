@@ -83,12 +83,18 @@ def load():
     lib.modse_check_device_status.argtypes = [vp, vp, vp]
     lib.modse_last_launch_count.restype = ci
     lib.modse_last_launch_count.argtypes = [vp]
+    lib.modse_debug_use_fma_path.restype = None
+    lib.modse_debug_use_fma_path.argtypes = [ci]
     _lib = lib
     return lib
 
 
 def status_string(status: int) -> str:
     return load().modse_status_string(int(status)).decode()
+
+
+def debug_use_fma_path(on: bool) -> None:
+    load().modse_debug_use_fma_path(int(bool(on)))
 
 
 def check_pairs(ffn_sizes):

@@ -370,4 +370,6 @@ modse_status_t modse_check_device_status(modse_layer_t *layer, const void *works
 
 int modse_last_launch_count(const modse_layer_t *layer) { return layer ? layer->last_launches : 0; }
 
+void modse_debug_use_fma_path(int on) { tc_set_force_simt(on); }
+
 }  // extern "C"

@@ -1,19 +1,11 @@
-#include <cstdlib>
-#include <cstring>
-
 #include "tc_gemm.h"
 
 namespace modse {
 
-bool tc_force_simt()
-{
-    static int v = -1;
-    if (v < 0) {
-        const char *e = std::getenv("MODSE_FORCE_SIMT");
-        v = (e != nullptr && std::strcmp(e, "1") == 0) ? 1 : 0;
-    }
-    return v == 1;
-}
+static int g_force_simt = 0;
+
+bool tc_force_simt() { return g_force_simt != 0; }
+void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
 
 modse_status_t tc_forward(TcPlan &, const LayerMeta &, const WsLayout &, const WsPtrs &, const modse_weights_t *,
                           bool, cudaStream_t, int *)

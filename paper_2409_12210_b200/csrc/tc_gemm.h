@@ -11,9 +11,10 @@ struct TcPlan {
     int dummy = 0;
 };
 
-// True when the environment asks for the fp32-FMA cross-check path
-// (MODSE_FORCE_SIMT=1); meant for debugging only.
+// Process-wide debugging switch: run bf16 layers through the fp32-FMA grouped
+// GEMMs instead of the tensor-core kernels.
 bool tc_force_simt();
+void tc_set_force_simt(int on);
 
 modse_status_t tc_forward(TcPlan &plan, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
                           const modse_weights_t *w, bool save, cudaStream_t s, int *launches);
