@@ -1,0 +1,90 @@
+"""GPU parity: the CUDA library through its C ABI against the fp64 oracle,
+element by element, at sizes the oracle finishes in seconds.
+
+Tolerances: routing tables bit-exact, gates 1e-6 absolute, every floating
+tensor max|err|/RMS(ref) <= 1e-4 for the fp32 type and <= 2e-2 for bf16."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+from paper_2409_12210_b200 import inputs as I
+
+import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+TOL_BF16 = 2e-2
+
+SMALL_BF16 = I.LayerConfig("small_bf16", "bf16", 256, (128, 384, 192, 320), 2, 300, seed=1)
+
+
+@pytest.fixture(scope="module", autouse=True)
+def lib():
+    from paper_2409_12210_b200 import build
+    build.build()
+
+
+def test_tiny_f32_forward_backward():
+    inp, _ = H.screened(I.CONFIGS["tiny_f32"])
+    gpu = H.run_gpu(inp, backward=True)
+    ora = H.run_oracle(inp, backward=True)
+    errs = H.check_all(inp, gpu, ora, TOL_F32)
+    assert gpu["launches_fwd"] > 0 and gpu["launches_bwd"] > 0, errs
+
+
+@pytest.mark.parametrize("T", [1, 63, 65, 257])
+def test_f32_ragged_token_counts(T):
+    inp, _ = H.screened(I.with_tokens(I.CONFIGS["tiny_f32"], T))
+    H.check_all(inp, H.run_gpu(inp, True), H.run_oracle(inp, True), TOL_F32)
+
+
+def test_f32_top1_and_single_expert_dense_ffn():
+    cfg = I.LayerConfig("top1", "f32", 64, (96, 160, 112, 144), 1, 100, seed=3)
+    inp, _ = H.screened(cfg)
+    gpu = H.run_gpu(inp, True)
+    H.check_all(inp, gpu, H.run_oracle(inp, True), TOL_F32)
+    assert np.all(gpu["routing"]["topk_gate"] == 1.0)
+    assert np.all(gpu["dw_router"] == 0.0)
+    dense = I.LayerConfig("dense", "f32", 64, (176,), 1, 70, seed=4)
+    inp = I.generate(dense)
+    H.check_all(inp, H.run_gpu(inp, True), H.run_oracle(inp, True), TOL_F32)
+
+
+def test_f32_exact_ties_go_to_lower_index_and_empty_expert():
+    inp, _ = H.screened(I.CONFIGS["tiny_f32"])
+    inp.w_router[3] = inp.w_router[1]                 # experts 1 and 3 tie exactly on every token
+    inp.x[5] = 0.0                                    # all logits equal: picks experts 0 and 1
+    gpu = H.run_gpu(inp, True)
+    ora = H.run_oracle(inp, True)
+    H.check_all(inp, gpu, ora, TOL_F32)
+    assert list(gpu["routing"]["topk_idx"][5]) == [0, 1]
+    # an expert nobody picks: its router row is far below the others
+    inp2, _ = H.screened(I.CONFIGS["tiny_f32"])
+    inp2.x = np.abs(inp2.x); inp2.w_router = np.abs(inp2.w_router); inp2.w_router[2] = -inp2.w_router[2]
+    gpu2 = H.run_gpu(inp2, True)
+    ora2 = H.run_oracle(inp2, True)
+    assert ora2["rt"].counts[2] == 0
+    H.check_all(inp2, gpu2, ora2, TOL_F32)
+    h0, h1 = sum(inp2.cfg.ffn_sizes[:2]), sum(inp2.cfg.ffn_sizes[:3])
+    assert np.all(gpu2["dw_gate"][h0:h1] == 0) and np.all(gpu2["dw_down"][:, h0:h1] == 0)
+
+
+def test_results_are_bitwise_reproducible():
+    inp, _ = H.screened(I.CONFIGS["tiny_f32"])
+    a = H.run_gpu(inp, True)
+    b = H.run_gpu(inp, True)
+    for k in ("y", "dx", "dw_router", "dw_gate", "dw_up", "dw_down", "dg", "dz"):
+        assert np.array_equal(a[k], b[k]), k
+
+
+def test_small_bf16_fma_cross_check_path():
+    from paper_2409_12210_b200 import binding as B
+    inp, _ = H.screened(SMALL_BF16)
+    B.debug_use_fma_path(True)
+    try:
+        gpu = H.run_gpu(inp, True)
+    finally:
+        B.debug_use_fma_path(False)
+    H.check_all(inp, gpu, H.run_oracle(inp, True), TOL_BF16)
