@@ -55,7 +55,7 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
     L.block_counts = take((size_t)L.nblk * m.k * N * 4);
     L.xp = take((size_t)L.Pmax * m.d * esz);
     L.hm = take(L.hb * esz);
-    L.o = take((size_t)L.Pmax * m.d * esz);
+    L.o = take((size_t)L.Pmax * m.d * 4);     // fp32 for every layer type
     if (save) {
         L.a_pre = take(L.hb * esz);
         L.b_pre = take(L.hb * esz);
@@ -65,7 +65,7 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
         L.dyp = take((size_t)L.Pmax * m.d * esz);
         L.da = take(L.hb * esz);
         L.db = take(L.hb * esz);
-        L.dxp = take((size_t)L.Pmax * m.d * esz);
+        L.dxp = take((size_t)L.Pmax * m.d * 4);   // fp32 for every layer type
     } else if (esz == 4) {
         // the fp32 path always materialises the two pre-activations
         L.a_pre = take(L.hb * esz);

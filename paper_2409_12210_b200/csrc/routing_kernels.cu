@@ -8,6 +8,9 @@
 //                      the stable destination row of every (token, slot).
 //   permute_kernel     gathers token rows into padded expert groups.
 //   combine_kernel     y_t = sum_j g[t,j] * o[row(t,j)]  (Sec. 3.1, Eq. 4).
+//                      (o and dxp, the two buffers that are summed over a
+//                      token's slots, are kept in fp32 for every layer type so
+//                      that the sum is rounded to the layer type only once.)
 //   dg_permute_kernel  dg[t,j] = <dY_t, o_(t,j)>, rows g*dY_t in group order.
 //   router_bwd_kernel  softmax Jacobian on the kept logits, dx assembly and
 //                      per-block partial sums of dW_router; reduced in block
@@ -306,7 +309,7 @@ permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int
 // ---------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
-combine_kernel(const T *__restrict__ o, int Ttok, int d, int k, const int *__restrict__ prow_of,
+combine_kernel(const float *__restrict__ o, int Ttok, int d, int k, const int *__restrict__ prow_of,
                const float *__restrict__ topk_gate, T *__restrict__ y)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -335,7 +338,7 @@ combine_kernel(const T *__restrict__ o, int Ttok, int d, int k, const int *__res
 // ---------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
-dg_permute_kernel(const T *__restrict__ dy, const T *__restrict__ o, int Ttok, int d, int N, int k,
+dg_permute_kernel(const T *__restrict__ dy, const float *__restrict__ o, int Ttok, int d, int N, int k,
                   const int *__restrict__ prow_of, const float *__restrict__ topk_gate,
                   const int *__restrict__ counts, const int *__restrict__ poffsets, float *__restrict__ dg,
                   T *__restrict__ dyp, int tok_blocks)
@@ -379,7 +382,8 @@ dg_permute_kernel(const T *__restrict__ dy, const T *__restrict__ o, int Ttok, i
 // ---------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
-router_bwd_kernel(const T *__restrict__ x, const T *__restrict__ w_router, const T *__restrict__ dxp, int Ttok,
+router_bwd_kernel(const T *__restrict__ x, const T *__restrict__ w_router, const float *__restrict__ dxp,
+                  int Ttok,
                   int d, int N, int k, int dc, const int *__restrict__ topk_idx,
                   const float *__restrict__ topk_gate, const int *__restrict__ prow_of,
                   const float *__restrict__ dg, float *__restrict__ dz, T *__restrict__ dx,
@@ -539,7 +543,7 @@ cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const Ws
         combine_kernel<float><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of, p.topk_gate,
                                                    (float *)y);
     else
-        combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)p.o, T, m.d, m.k, p.prow_of,
+        combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of,
                                                            p.topk_gate, (__nv_bfloat16 *)y);
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
@@ -556,7 +560,7 @@ cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *
                                                       (float *)p.dyp, tok_blocks);
     else
         dg_permute_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)dy,
-                                                              (const __nv_bfloat16 *)p.o, T, m.d, m.N, m.k,
+                                                              (const float *)p.o, T, m.d, m.N, m.k,
                                                               p.prow_of, p.topk_gate, p.counts, p.poffsets, p.dg,
                                                               (__nv_bfloat16 *)p.dyp, tok_blocks);
     MODSE_LAUNCH_CHECK();
@@ -586,7 +590,7 @@ cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<grid, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router,
-                                     (const __nv_bfloat16 *)p.dxp, T, m.d, m.N, m.k, dc, p.topk_idx, p.topk_gate,
+                                     (const float *)p.dxp, T, m.d, m.N, m.k, dc, p.topk_idx, p.topk_gate,
                                      p.prow_of, p.dg, p.dz, (__nv_bfloat16 *)dx, p.dwr_partial);
     }
     MODSE_LAUNCH_CHECK();

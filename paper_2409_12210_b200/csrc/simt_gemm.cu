@@ -25,14 +25,20 @@ __device__ __forceinline__ float ld(const __nv_bfloat16 *p, long long i) { retur
 __device__ __forceinline__ void st(float *p, long long i, float v) { p[i] = v; }
 __device__ __forceinline__ void st(__nv_bfloat16 *p, long long i, float v) { p[i] = __float2bfloat16_rn(v); }
 
+// Results that are later summed over a token's slots (o of kDown, dxp of
+// kUpGateDgrad) are fp32 buffers whatever the layer type.
+__host__ __device__ inline bool out_is_f32(int kind) { return kind == kDown || kind == kUpGateDgrad; }
+
 template <typename T>
 __device__ Problem make_problem(int kind, const LayerMeta &m, int e, const int *poffsets, const long long *ebase,
-                                const T *act, const T *wgt, T *out)
+                                const T *act, const T *wgt, void *out_v)
 {
     const long long d = m.d, S = m.S;
     const long long ho = m.hoff[e], he = m.hoff[e + 1] - m.hoff[e];
     const long long po = poffsets[e], cp = poffsets[e + 1] - poffsets[e];
     const long long eb = ebase[e];
+    T *out = static_cast<T *>(out_v);
+    float *outf = static_cast<float *>(out_v);
     Problem p;
     switch (kind) {
     case kUpGate:       // C[cp,he] = xp . W^T
@@ -43,7 +49,7 @@ __device__ Problem make_problem(int kind, const LayerMeta &m, int e, const int *
     case kDown:         // o[cp,d] = Hm . W_down_e^T, W_down is [d,S]
         p.A = act + eb; p.a_rs = he; p.a_cs = 1;
         p.B = wgt + ho; p.b_rs = S; p.b_cs = 1;
-        p.C = out + po * d; p.c_rs = d; p.M = (int)cp; p.Nn = (int)d; p.K = (int)he;
+        p.C = outf + po * d; p.c_rs = d; p.M = (int)cp; p.Nn = (int)d; p.K = (int)he;
         break;
     case kDownDgrad:    // dHm[cp,he] = dyp . W_down_e ; B(n,k) = W_down[k, ho+n]
         p.A = act + po * d; p.a_rs = d; p.a_cs = 1;
@@ -58,7 +64,7 @@ __device__ Problem make_problem(int kind, const LayerMeta &m, int e, const int *
     case kUpGateDgrad:  // dxp[cp,d] (+)= dA . W ; B(n,k) = W[ho+k, n]
         p.A = act + eb; p.a_rs = he; p.a_cs = 1;
         p.B = wgt + ho * d; p.b_rs = 1; p.b_cs = d;
-        p.C = out + po * d; p.c_rs = d; p.M = (int)cp; p.Nn = (int)d; p.K = (int)he;
+        p.C = outf + po * d; p.c_rs = d; p.M = (int)cp; p.Nn = (int)d; p.K = (int)he;
         break;
     default:            // kUpGateWgrad: dW[ho+r, c] = sum_i dA[i,r] xp[i,c]
         p.A = act + eb; p.a_rs = 1; p.a_cs = he;
@@ -74,7 +80,7 @@ constexpr int BM = 64, BN = 64, BK = 16;
 template <typename T>
 __global__ void __launch_bounds__(256)
 simt_grouped_gemm(int kind, LayerMeta m, const int *__restrict__ poffsets, const long long *__restrict__ ebase,
-                  const T *act, const T *wgt, T *out, int accumulate)
+                  const T *act, const T *wgt, void *out, int accumulate)
 {
     const int e = blockIdx.z;
     const Problem p = make_problem<T>(kind, m, e, poffsets, ebase, act, wgt, out);
@@ -85,6 +91,8 @@ simt_grouped_gemm(int kind, LayerMeta m, const int *__restrict__ poffsets, const
     const T *A = static_cast<const T *>(p.A);
     const T *B = static_cast<const T *>(p.B);
     T *C = static_cast<T *>(p.C);
+    float *Cf = static_cast<float *>(p.C);
+    const bool f32out = out_is_f32(kind);
     const int tid = threadIdx.x;
     const int tx = tid % 16, ty = tid / 16;
     float acc[4][4] = {};
@@ -128,8 +136,13 @@ simt_grouped_gemm(int kind, LayerMeta m, const int *__restrict__ poffsets, const
             if (nn >= p.Nn) continue;
             const long long idx = (long long)mm * p.c_rs + nn;
             float v = acc[i][j];
-            if (accumulate) v += ld(C, idx);
-            st(C, idx, v);
+            if (f32out) {
+                if (accumulate) v += Cf[idx];
+                Cf[idx] = v;
+            } else {
+                if (accumulate) v += ld(C, idx);
+                st(C, idx, v);
+            }
         }
     }
 }
@@ -181,12 +194,11 @@ cudaError_t launch_simt_gemm(modse_dtype_t dt, GemmKind kind, const LayerMeta &m
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
     if (dt == MODSE_F32)
         simt_grouped_gemm<float><<<grid, 256, 0, s>>>((int)kind, m, p.poffsets, p.ebase, (const float *)a.act,
-                                                      (const float *)a.wgt, (float *)a.out, a.accumulate);
+                                                      (const float *)a.wgt, a.out, a.accumulate);
     else
         simt_grouped_gemm<__nv_bfloat16><<<grid, 256, 0, s>>>((int)kind, m, p.poffsets, p.ebase,
                                                               (const __nv_bfloat16 *)a.act,
-                                                              (const __nv_bfloat16 *)a.wgt, (__nv_bfloat16 *)a.out,
-                                                              a.accumulate);
+                                                              (const __nv_bfloat16 *)a.wgt, a.out, a.accumulate);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (launches) ++*launches;
