@@ -1,22 +1,721 @@
+// Grouped GEMMs of the bf16 MoDSE layer on Blackwell tensor cores.
+//
+// One persistent, warp-specialised kernel template serves the six products of
+// the layer (Sec. 3.1, Eq. 4 and its gradient); a tile is 128 rows by up to 256
+// fp32 accumulator columns held in tensor memory (TMEM):
+//
+//   kind            product (per expert e, cp = padded rows, h = width)      K
+//   UpGate          Hm = silu(xp Wg^T) * (xp Wu^T)          [cp, h]          d
+//   Down            o  = Hm Wd_e^T                          [cp, d]  fp32    h
+//   DownDgrad       dHm = dyp Wd_e -> dA, dB (SwiGLU bwd)   [cp, h]          d
+//   DownWgrad       dWd_e = dyp^T Hm                        [d, h]           cp
+//   UpGateDgrad     dxp = dA Wg_e + dB Wu_e                 [cp, d]  fp32    2h
+//   UpGateWgrad     dWg_e = dA^T xp, dWu_e = dB^T xp        [h, d]           cp
+//
+// Roles inside a CTA (192 threads): warp 0 issues TMA loads into a 4-stage
+// shared-memory ring (every box is 64 elements x 64 rows, 128-byte swizzle),
+// warp 1 issues tcgen05.mma with the accumulator in TMEM (two accumulators, so
+// the epilogue of one tile overlaps the main loop of the next), warps 2-5 read
+// the accumulator with tcgen05.ld and run the fused epilogue.  Operands are
+// consumed either K-major or MN-major straight from their row-major buffers
+// (the instruction descriptor carries the major-ness), so the backward pass
+// needs no transposed copies.
+//
+// Activations that have the hidden axis as their width (Hm, the saved
+// pre-activations, dA, dB) are stored as panels: for expert e, panel pc holds
+// columns [64 pc, 64 pc + 64) of all cp rows contiguously, so that a single
+// two-dimensional tensor map with 128-byte rows describes the whole buffer
+// although the row length h differs from expert to expert.
+//
+// Tiles are handed out statically: experts are ordered by decreasing K so the
+// long tiles of wide experts (or of experts with many tokens) start first and
+// the short ones fill the tail - the one-GPU form of the paper's expert-pair
+// balancing (Sec. 3.2).  Every wait is bounded; a wait that expires records
+// kDevTimeout in the status word and the CTA drains and exits.
+#include <cuda.h>
+
 #include "tc_gemm.h"
 
 namespace modse {
 
 static int g_force_simt = 0;
-
 bool tc_force_simt() { return g_force_simt != 0; }
 void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
 
-modse_status_t tc_forward(TcPlan &, const LayerMeta &, const WsLayout &, const WsPtrs &, const modse_weights_t *,
-                          bool, cudaStream_t, int *)
+namespace {
+
+enum TcKind : int { TcUpGate = 0, TcDown = 1, TcDownDgrad = 2, TcDownWgrad = 3, TcUpGateDgrad = 4, TcUpGateWgrad = 5 };
+
+constexpr int kStages = 4;
+constexpr int kBoxBytes = 64 * 64 * 2;           // one TMA box: 64 rows of 128 bytes
+constexpr int kARegion = 2 * kBoxBytes;          // 128 rows (or 128 MN elements) x 64 K
+constexpr int kBRegion = 4 * kBoxBytes;          // up to 256 rows x 64 K
+constexpr int kStageBytes = kARegion + kBRegion; // 48 KB
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr int kAccCols = 256;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+
+struct TcMaps {
+    CUtensorMap xp, dyp, wgate, wup, wdown, hm, da, db;
+};
+
+struct TcParams {
+    LayerMeta meta;
+    const int *poffsets;
+    const long long *ebase;
+    int *status;
+    __nv_bfloat16 *hm, *a_pre, *b_pre, *da, *db;
+    float *o, *dxp;
+    __nv_bfloat16 *dw_gate, *dw_up, *dw_down;
+    int save;
+};
+
+// dynamic shared memory map (after 1024-byte alignment)
+struct SmemTail {
+    unsigned long long full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+    unsigned int tmem_base;
+    int abort_flag;
+    int order[kMaxExperts];
+    int key[kMaxExperts];
+    int ntile[kMaxExperts];
+    int tstart[kMaxExperts + 1];
+};
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(SmemTail);
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    return MODSE_ERR_UNSUPPORTED;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false if the phase did not complete within kWaitLimitNs or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    unsigned it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 255u) == 0) {
+            if (*abort_flag || global_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicMax(status, kDevTimeout);
+                return false;
+            }
+        }
+    }
+    return true;
 }
 
-modse_status_t tc_backward(TcPlan &, const LayerMeta &, const WsLayout &, const WsPtrs &, const modse_weights_t *,
-                           const modse_wgrads_t *, cudaStream_t, int *)
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
 {
-    return MODSE_ERR_UNSUPPORTED;
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), version 1.
+//   K-major : rows of 128 bytes, 8-row groups 1024 bytes apart (SBO); LBO unused.
+//   MN-major: k-rows of 128 bytes holding 64 MN elements, 8-k groups 1024 bytes
+//             apart (SBO), 64-element MN blocks 8192 bytes apart (LBO).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major)
+{
+    const uint64_t lbo = mn_major ? (uint64_t)(kBoxBytes >> 4) : 1ull;
+    const uint64_t sbo = 1024 >> 4;
+    return (uint64_t)((saddr & 0x3FFFF) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
+}
+
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128.
+__device__ __forceinline__ uint32_t make_idesc(bool a_mn, bool b_mn, int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+template <int KIND> struct KindTraits;
+template <> struct KindTraits<TcUpGate>      { static constexpr bool a_mn = false, b_mn = false; };
+template <> struct KindTraits<TcDown>        { static constexpr bool a_mn = false, b_mn = false; };
+template <> struct KindTraits<TcDownDgrad>   { static constexpr bool a_mn = false, b_mn = true; };
+template <> struct KindTraits<TcDownWgrad>   { static constexpr bool a_mn = true,  b_mn = true; };
+template <> struct KindTraits<TcUpGateDgrad> { static constexpr bool a_mn = false, b_mn = true; };
+template <> struct KindTraits<TcUpGateWgrad> { static constexpr bool a_mn = true,  b_mn = true; };
+
+struct Tile {
+    int e, cp, h, ho, prow0, pbase;   // expert, padded rows, width, width offset, first padded row, first panel row
+    int m0, n0, mrows, ncols, nk, which;
+    int n_mma, a_boxes, b_boxes;
+};
+
+// tiles (rows, columns) and K blocks of one expert
+template <int KIND>
+__device__ __forceinline__ void expert_shape(int cp, int h, int d, int &mt, int &nt, int &nk)
+{
+    if constexpr (KIND == TcUpGate)      { mt = cp / 128; nt = (h + 127) / 128; nk = d / 64; }
+    if constexpr (KIND == TcDown)        { mt = cp / 128; nt = (d + 255) / 256; nk = h / 64; }
+    if constexpr (KIND == TcDownDgrad)   { mt = cp / 128; nt = (h + 255) / 256; nk = d / 64; }
+    if constexpr (KIND == TcDownWgrad)   { mt = d / 128;  nt = (h + 255) / 256; nk = cp / 64; }
+    if constexpr (KIND == TcUpGateDgrad) { mt = cp / 128; nt = (d + 255) / 256; nk = 2 * (h / 64); }
+    if constexpr (KIND == TcUpGateWgrad) { mt = 2 * ((h + 127) / 128); nt = (d + 255) / 256; nk = cp / 64; }
+}
+
+template <int KIND>
+__device__ __forceinline__ Tile decode_tile(const TcParams &prm, const SmemTail *st, int tile, int &cursor)
+{
+    const int N = prm.meta.N, d = prm.meta.d;
+    while (cursor + 1 < N && tile >= st->tstart[cursor + 1]) ++cursor;
+    Tile t;
+    t.e = st->order[cursor];
+    t.ho = prm.meta.hoff[t.e];
+    t.h = prm.meta.hoff[t.e + 1] - t.ho;
+    t.prow0 = prm.poffsets[t.e];
+    t.cp = prm.poffsets[t.e + 1] - t.prow0;
+    t.pbase = (int)(prm.ebase[t.e] >> 6);
+    int mt, nt, nk;
+    expert_shape<KIND>(t.cp, t.h, d, mt, nt, nk);
+    const int local = tile - st->tstart[cursor];
+    const int mb = local % mt, nb = local / mt;
+    t.nk = nk;
+    t.which = 0;
+    t.mrows = 128;
+    if constexpr (KIND == TcUpGate) {
+        t.m0 = mb * 128; t.n0 = nb * 128; t.ncols = min(128, t.h - t.n0);
+        t.n_mma = 2 * t.ncols; t.a_boxes = 2; t.b_boxes = t.n_mma / 64;
+    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
+        t.m0 = mb * 128; t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
+        t.n_mma = t.ncols; t.a_boxes = 2; t.b_boxes = t.ncols / 64;
+    } else if constexpr (KIND == TcDownDgrad || KIND == TcDownWgrad) {
+        t.m0 = mb * 128; t.n0 = nb * 256; t.ncols = min(256, t.h - t.n0);
+        t.n_mma = t.ncols; t.a_boxes = 2; t.b_boxes = t.ncols / 64;
+    } else {
+        t.which = mb & 1;
+        t.m0 = (mb >> 1) * 128; t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
+        t.mrows = min(128, t.h - t.m0);
+        t.n_mma = t.ncols; t.a_boxes = t.mrows / 64; t.b_boxes = t.ncols / 64;
+    }
+    return t;
+}
+
+// TMA loads of k-block kb of a tile into one stage.
+template <int KIND>
+__device__ __forceinline__ void issue_loads(const TcMaps &maps, const Tile &t, int kb, uint32_t a_dst, uint32_t b_dst,
+                                            uint32_t bar)
+{
+    if constexpr (KIND == TcUpGate) {
+        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, &maps.xp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        const int nb = t.ncols / 64;
+        for (int i = 0; i < nb; ++i) tma_load_2d(b_dst + i * kBoxBytes, &maps.wgate, bar, kb * 64, t.ho + t.n0 + 64 * i);
+        for (int i = 0; i < nb; ++i)
+            tma_load_2d(b_dst + (nb + i) * kBoxBytes, &maps.wup, bar, kb * 64, t.ho + t.n0 + 64 * i);
+    } else if constexpr (KIND == TcDown) {
+        for (int i = 0; i < 2; ++i)
+            tma_load_2d(a_dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + kb * t.cp + t.m0 + 64 * i);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + kb * 64, t.n0 + 64 * i);
+    } else if constexpr (KIND == TcDownDgrad) {
+        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, &maps.dyp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + 64 * i, kb * 64);
+    } else if constexpr (KIND == TcDownWgrad) {
+        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d(b_dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + (t.n0 / 64 + i) * t.cp + kb * 64);
+    } else if constexpr (KIND == TcUpGateDgrad) {
+        const int half = t.h / 64;
+        const bool second = kb >= half;
+        const int kk = second ? kb - half : kb;
+        const CUtensorMap *am = second ? &maps.db : &maps.da;
+        const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
+        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + kk * t.cp + t.m0 + 64 * i);
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(b_dst + i * kBoxBytes, bm, bar, t.n0 + 64 * i, t.ho + kk * 64);
+    } else {
+        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d(b_dst + i * kBoxBytes, &maps.xp, bar, t.n0 + 64 * i, t.prow0 + kb * 64);
+    }
+}
+
+__device__ __forceinline__ void store_bf16x32(__nv_bfloat16 *dst, const float (&v)[32])
+{
+    uint4 *p = reinterpret_cast<uint4 *>(dst);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t *>(&t);
+        }
+        p[q] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+__device__ __forceinline__ void load_bf16x32(const __nv_bfloat16 *src, float (&v)[32])
+{
+    const uint4 *p = reinterpret_cast<const uint4 *>(src);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        const uint4 u = p[q];
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[q * 8 + 2 * i] = __uint_as_float(w[i] << 16);
+            v[q * 8 + 2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+}
+
+__device__ __forceinline__ void store_f32x32(float *dst, const float (&v)[32])
+{
+    float4 *p = reinterpret_cast<float4 *>(dst);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) p[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+}
+
+// Epilogue of one tile for one thread (= one accumulator row).
+template <int KIND>
+__device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t, uint32_t tacc, int row)
+{
+    const int d = prm.meta.d, S = prm.meta.S;
+    const bool have_acc = t.nk > 0;
+    if constexpr (KIND == TcUpGate) {
+        for (int c = 0; c < t.ncols; c += 32) {
+            uint32_t ra[32], rb[32];
+            tmem_ld32(tacc + c, ra);
+            tmem_ld32(tacc + t.ncols + c, rb);
+            tmem_ld_wait();
+            float hm[32], av[32], bv[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                av[i] = __uint_as_float(ra[i]);
+                bv[i] = __uint_as_float(rb[i]);
+                hm[i] = av[i] * (1.0f / (1.0f + __expf(-av[i]))) * bv[i];
+            }
+            const int col = t.n0 + c;
+            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
+            store_bf16x32(prm.hm + idx, hm);
+            if (prm.save) {
+                store_bf16x32(prm.a_pre + idx, av);
+                store_bf16x32(prm.b_pre + idx, bv);
+            }
+        }
+    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
+        float *out = (KIND == TcDown ? prm.o : prm.dxp) + (size_t)(t.prow0 + t.m0 + row) * d + t.n0;
+        for (int c = 0; c < t.ncols; c += 32) {
+            uint32_t r[32];
+            float v[32];
+            tmem_ld32(tacc + c, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+            store_f32x32(out + c, v);
+        }
+    } else if constexpr (KIND == TcDownDgrad) {
+        for (int c = 0; c < t.ncols; c += 32) {
+            uint32_t r[32];
+            tmem_ld32(tacc + c, r);
+            tmem_ld_wait();
+            const int col = t.n0 + c;
+            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
+            float av[32], bv[32], da[32], db[32];
+            load_bf16x32(prm.a_pre + idx, av);
+            load_bf16x32(prm.b_pre + idx, bv);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float dh = __uint_as_float(r[i]);
+                const float sg = 1.0f / (1.0f + __expf(-av[i]));
+                da[i] = dh * bv[i] * sg * (1.0f + av[i] * (1.0f - sg));
+                db[i] = dh * av[i] * sg;
+            }
+            store_bf16x32(prm.da + idx, da);
+            store_bf16x32(prm.db + idx, db);
+        }
+    } else if constexpr (KIND == TcDownWgrad) {
+        __nv_bfloat16 *out = prm.dw_down + (size_t)(t.m0 + row) * S + t.ho + t.n0;
+        for (int c = 0; c < t.ncols; c += 32) {
+            float v[32];
+            if (have_acc) {
+                uint32_t r[32];
+                tmem_ld32(tacc + c, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = 0.f;
+            }
+            store_bf16x32(out + c, v);
+        }
+    } else {
+        __nv_bfloat16 *out = (t.which ? prm.dw_up : prm.dw_gate) + (size_t)(t.ho + t.m0 + row) * d + t.n0;
+        for (int c = 0; c < t.ncols; c += 32) {
+            float v[32];
+            if (have_acc) {
+                uint32_t r[32];
+                tmem_ld32(tacc + c, r);      // whole warp takes part in the load, also for rows that are not stored
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = 0.f;
+            }
+            if (row < t.mrows) store_bf16x32(out + c, v);
+        }
+    }
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
+    unsigned char *smem = smem_raw + pad;
+    const uint32_t stage_base = raw + pad;
+    SmemTail *st = reinterpret_cast<SmemTail *>(smem + (size_t)kStages * kStageBytes);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int N = prm.meta.N, d = prm.meta.d;
+
+    // ---- schedule: experts by decreasing K, tiles of an expert contiguous ----
+    for (int e = tid; e < N; e += kThreads) {
+        const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
+        const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
+        int mt, nt, nk;
+        expert_shape<KIND>(cp, h, d, mt, nt, nk);
+        st->ntile[e] = mt * nt;
+        st->key[e] = nk;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&st->full[s]), 1);
+            mbar_init(smem_u32(&st->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&st->tmem_full[a]), 1);
+            mbar_init(smem_u32(&st->tmem_empty[a]), 128);
+        }
+        st->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    for (int e = tid; e < N; e += kThreads) {
+        int rank = 0;
+        const int ke = st->key[e];
+        for (int f = 0; f < N; ++f) {
+            const int kf = st->key[f];
+            rank += (kf > ke) || (kf == ke && f < e);
+        }
+        st->order[rank] = e;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&st->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int i = 0; i < N; ++i) { st->tstart[i] = acc; acc += st->ntile[st->order[i]]; }
+        st->tstart[N] = acc;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = st->tmem_base;
+    const int total_tiles = st->tstart[N];
+    volatile int *abort_flag = &st->abort_flag;
+
+    if (warp == 0) {
+        // ===================== TMA producer =====================
+        if (lane == 0) {
+            int stage = 0, cursor = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const Tile t = decode_tile<KIND>(prm, st, tile, cursor);
+                const uint32_t bytes = (uint32_t)(t.a_boxes + t.b_boxes) * kBoxBytes;
+                for (int kb = 0; kb < t.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&st->full[stage]);
+                    mbar_arrive_expect_tx(bar, bytes);
+                    const uint32_t a_dst = stage_base + stage * kStageBytes;
+                    issue_loads<KIND>(maps, t, kb, a_dst, a_dst + kARegion, bar);
+                    ++issued;
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // let the copies already issued land before the CTA leaves: wait (bounded) for
+                // the current phase of every stage that has had a load
+                const int n = issued < kStages ? (int)issued : kStages;
+                for (int i = 1; i <= n; ++i) {
+                    int s = stage - i;
+                    uint32_t ph = phase;
+                    if (s < 0) { s += kStages; ph ^= 1u; }
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(smem_u32(&st->full[s]), ph) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===================== MMA issuer =====================
+        if (lane == 0) {
+            int stage = 0, cursor = 0, it = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            constexpr bool a_mn = KindTraits<KIND>::a_mn, b_mn = KindTraits<KIND>::b_mn;
+            constexpr uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
+            constexpr uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+                const Tile t = decode_tile<KIND>(prm, st, tile, cursor);
+                const int acc = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + (uint32_t)(acc * kAccCols);
+                const uint32_t idesc = make_idesc(a_mn, b_mn, t.n_mma);
+                for (int kb = 0; kb < t.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->full[stage]), phase, abort_flag, prm.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stage_base + stage * kStageBytes;
+                    const uint64_t adesc = make_desc(a_addr, a_mn);
+                    const uint64_t bdesc = make_desc(a_addr + kARegion, b_mn);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_bf16(tacc, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
+                                  (kb > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit(smem_u32(&st->empty[stage]));   // frees the stage once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (t.nk > 0) umma_commit(smem_u32(&st->tmem_full[acc]));
+                else mbar_arrive(smem_u32(&st->tmem_full[acc]));
+            }
+        }
+    } else {
+        // ===================== epilogue (warps 2..5) =====================
+        const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+        const int row = quad * 32 + lane;
+        int cursor = 0, it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+            const Tile t = decode_tile<KIND>(prm, st, tile, cursor);
+            const int acc = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, prm.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
+            epilogue_row<KIND>(prm, t, tacc, row);
+            tc_fence_before();
+            mbar_arrive(smem_u32(&st->tmem_empty[acc]));
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 row-major matrix [rows, cols] seen as a 2-D tensor, 64 x 64 boxes, 128-byte swizzle.
+bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols)
+{
+    EncodeTiledFn fn = get_encode();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {64, 64};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
+               bool backward)
+{
+    const uint64_t panel_rows = L.hb / 64;
+    bool ok = true;
+    ok = ok && encode_2d(&maps.xp, p.xp, L.Pmax, m.d);
+    ok = ok && encode_2d(&maps.wgate, w->w_gate, m.S, m.d);
+    ok = ok && encode_2d(&maps.wup, w->w_up, m.S, m.d);
+    ok = ok && encode_2d(&maps.wdown, w->w_down, m.d, m.S);
+    ok = ok && encode_2d(&maps.hm, p.hm, panel_rows, 64);
+    if (backward) {
+        ok = ok && encode_2d(&maps.dyp, p.dyp, L.Pmax, m.d);
+        ok = ok && encode_2d(&maps.da, p.da, panel_rows, 64);
+        ok = ok && encode_2d(&maps.db, p.db, panel_rows, 64);
+    } else {
+        maps.dyp = maps.xp;
+        maps.da = maps.hm;
+        maps.db = maps.hm;
+    }
+    return ok;
+}
+
+TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *g, bool save)
+{
+    TcParams prm{};
+    prm.meta = m;
+    prm.poffsets = p.poffsets;
+    prm.ebase = p.ebase;
+    prm.status = p.status;
+    prm.hm = (__nv_bfloat16 *)p.hm;
+    prm.a_pre = (__nv_bfloat16 *)p.a_pre;
+    prm.b_pre = (__nv_bfloat16 *)p.b_pre;
+    prm.da = (__nv_bfloat16 *)p.da;
+    prm.db = (__nv_bfloat16 *)p.db;
+    prm.o = (float *)p.o;
+    prm.dxp = (float *)p.dxp;
+    if (g) {
+        prm.dw_gate = (__nv_bfloat16 *)g->dw_gate;
+        prm.dw_up = (__nv_bfloat16 *)g->dw_up;
+        prm.dw_down = (__nv_bfloat16 *)g->dw_down;
+    }
+    prm.save = save ? 1 : 0;
+    return prm;
+}
+
+template <int KIND>
+cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
+{
+    auto kern = tc_grouped_gemm<KIND>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, kSmemBytes, s>>>(maps, prm);
+    e = cudaGetLastError();
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+int sm_count(TcPlan &plan)
+{
+    if (plan.sm_count == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            plan.sm_count = n;
+        else
+            plan.sm_count = 148;
+    }
+    return plan.sm_count;
+}
+
+}  // namespace
+
+modse_status_t tc_forward(TcPlan &plan, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
+                          const modse_weights_t *w, bool save, cudaStream_t s, int *launches)
+{
+    TcMaps maps;
+    if (!fill_maps(maps, m, L, p, w, false)) return MODSE_ERR_CUDA;
+    const TcParams prm = make_params(m, p, nullptr, save);
+    const int grid = sm_count(plan);
+    if (launch_kind<TcUpGate>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (launch_kind<TcDown>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
+    return MODSE_OK;
+}
+
+modse_status_t tc_backward(TcPlan &plan, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
+                           const modse_weights_t *w, const modse_wgrads_t *g, cudaStream_t s, int *launches)
+{
+    TcMaps maps;
+    if (!fill_maps(maps, m, L, p, w, true)) return MODSE_ERR_CUDA;
+    const TcParams prm = make_params(m, p, g, true);
+    const int grid = sm_count(plan);
+    if (launch_kind<TcDownDgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (launch_kind<TcDownWgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (launch_kind<TcUpGateDgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (launch_kind<TcUpGateWgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
+    return MODSE_OK;
 }
 
 }  // namespace modse

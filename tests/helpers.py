@@ -27,6 +27,19 @@ def rel_err(got, ref) -> float:
     return float(np.max(np.abs(got - ref)) / rms)
 
 
+def rel_err_beyond_storage(got, ref) -> float:
+    """Like rel_err, but the part of each element's error that one bf16 rounding of the
+    stored result explains (at most 2^-8 |ref|) is not counted.  For heavy-tailed tensors
+    (weight gradients summed over a handful of tokens) that rounding alone exceeds any
+    RMS-relative bound, whatever computed the value."""
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    if not ref.size:
+        return 0.0
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    excess = np.maximum(0.0, np.abs(got - ref) - np.abs(ref) * 2.0 ** -8)
+    return float(excess.max() / rms) if rms > 0 else float(excess.max())
+
+
 def run_gpu(inp: I.LayerInputs, backward: bool, save: bool | None = None):
     """Forward (and backward) through the C ABI; returns host numpy results."""
     import torch
@@ -80,21 +93,25 @@ def check_routing(gpu_rt, rt, gate_tol=1e-6):
     assert np.max(np.abs(gpu_rt["topk_gate"] - rt.topk_gate)) <= gate_tol
 
 
-def check_all(inp, gpu, ora, tol):
-    """Element-by-element comparison of every output; returns the error table."""
+def check_all(inp, gpu, ora, tol, discount_storage_rounding=False):
+    """Element-by-element comparison of every output; returns the error table.
+    With discount_storage_rounding the bf16-stored tensors are measured with
+    rel_err_beyond_storage (degenerate shapes only)."""
     check_routing(gpu["routing"], ora["rt"])
-    errs = {"y": rel_err(gpu["y"], ora["y"])}
+    full = rel_err
+    rel_err_ = rel_err_beyond_storage if discount_storage_rounding else rel_err
+    errs = {"y": rel_err_(gpu["y"], ora["y"])}
     if "dx" in gpu:
         g = ora["g"]
         rt = ora["rt"]
-        errs["dx"] = rel_err(gpu["dx"], g.dx)
-        errs["dw_router"] = rel_err(gpu["dw_router"], g.dw_router)
-        errs["dw_gate"] = rel_err(gpu["dw_gate"], np.concatenate(g.dw_gate, 0))
-        errs["dw_up"] = rel_err(gpu["dw_up"], np.concatenate(g.dw_up, 0))
-        errs["dw_down"] = rel_err(gpu["dw_down"], np.concatenate(g.dw_down, 1))
-        errs["dg"] = rel_err(gpu["dg"], g.dg)
+        errs["dx"] = rel_err_(gpu["dx"], g.dx)
+        errs["dw_router"] = full(gpu["dw_router"], g.dw_router)
+        errs["dw_gate"] = rel_err_(gpu["dw_gate"], np.concatenate(g.dw_gate, 0))
+        errs["dw_up"] = rel_err_(gpu["dw_up"], np.concatenate(g.dw_up, 0))
+        errs["dw_down"] = rel_err_(gpu["dw_down"], np.concatenate(g.dw_down, 1))
+        errs["dg"] = full(gpu["dg"], g.dg)
         dz_kept = np.take_along_axis(g.dz, rt.topk_idx.astype(np.int64), 1)
-        errs["dz"] = rel_err(gpu["dz"], dz_kept)
+        errs["dz"] = full(gpu["dz"], dz_kept)
     assert gpu["status"] == 0
     bad = {k: v for k, v in errs.items() if not (v <= tol)}
     assert not bad, f"over tolerance {tol}: {bad} (all: {errs})"

@@ -17,7 +17,8 @@ pytestmark = pytest.mark.gpu
 TOL_F32 = 1e-4
 TOL_BF16 = 2e-2
 
-SMALL_BF16 = I.LayerConfig("small_bf16", "bf16", 256, (128, 384, 192, 320), 2, 300, seed=1)
+# 1000 tokens: every expert group spans several 128-row tiles and ends in a ragged one
+SMALL_BF16 = I.LayerConfig("small_bf16", "bf16", 256, (128, 384, 192, 320), 2, 1000, seed=1, weight_std=0.05)
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -80,6 +81,8 @@ def test_results_are_bitwise_reproducible():
 
 
 def test_small_bf16_fma_cross_check_path():
+    # the debugging path rounds the pre-activations and dHm to bf16 on the way, so it is
+    # held to the bound only beyond storage rounding
     from paper_2409_12210_b200 import binding as B
     inp, _ = H.screened(SMALL_BF16)
     B.debug_use_fma_path(True)
@@ -87,4 +90,27 @@ def test_small_bf16_fma_cross_check_path():
         gpu = H.run_gpu(inp, True)
     finally:
         B.debug_use_fma_path(False)
+    H.check_all(inp, gpu, H.run_oracle(inp, True), TOL_BF16, discount_storage_rounding=True)
+
+
+def test_small_bf16_tensor_core_path():
+    inp, _ = H.screened(SMALL_BF16)
+    gpu = H.run_gpu(inp, True)
     H.check_all(inp, gpu, H.run_oracle(inp, True), TOL_BF16)
+
+
+def test_small_bf16_forward_only_without_saving():
+    inp, _ = H.screened(SMALL_BF16)
+    gpu = H.run_gpu(inp, False)
+    H.check_all(inp, gpu, H.run_oracle(inp, False), TOL_BF16)
+
+
+@pytest.mark.parametrize("T,k,widths,d", [(1, 2, (64, 128), 128), (129, 1, (64, 192, 128), 128),
+                                          (700, 2, (448, 64, 320, 192), 384)])
+def test_bf16_degenerate_and_ragged_shapes(T, k, widths, d):
+    # With a handful of tokens per expert the weight gradients are heavy-tailed and one bf16
+    # rounding of the stored value (2^-8 |v|) alone passes 2e-2 RMS; that share is discounted here.
+    cfg = I.LayerConfig(f"bf16_T{T}", "bf16", d, widths, k, T, seed=T)
+    inp, _ = H.screened(cfg)
+    gpu = H.run_gpu(inp, True)
+    H.check_all(inp, gpu, H.run_oracle(inp, True), TOL_BF16, discount_storage_rounding=True)
