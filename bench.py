@@ -1,0 +1,337 @@
+"""Benchmark of the MoDSE layer (forward + backward) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One step is one pass of the whole layer - router, permutation, grouped up/gate
+GEMM with SwiGLU, grouped down GEMM, combine, and the full backward - over one
+batch of seeded synthetic tokens shaped like the paper's 700M x 8 model (width
+2048, 8 experts, top-2).  Prints ONE JSON line.
+
+N > 1 runs N independent replicas of the layer (one process per GPU under
+torchrun): the layer runs on one GPU and has no exchange step, so throughput is
+reported as weak scaling over replicas, timed as the maximum over ranks.
+
+`--impl reference` times the fp64 CPU checker (the only other implementation
+of this layer) on a bounded sample of the same workload, on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2409_12210_b200 import inputs as I  # noqa: E402
+
+METRIC = "modse_layer_fwd_bwd_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+STAGE_BOUND = ["hbm", "hbm", "hbm", "tensor", "tensor", "hbm", "hbm", "tensor", "tensor", "tensor", "tensor", "hbm"]
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def expert_flops(counts, cfg):
+    """Algorithmic FLOPs of the expert GEMMs for the measured routing histogram:
+    forward sum_e c_e * 6 d h_e, backward twice that; router 2TdN forward, 4TdN backward."""
+    d, T, N = cfg.d_model, cfg.n_tokens, cfg.n_experts
+    ch = float(sum(int(c) * h for c, h in zip(counts, cfg.ffn_sizes)))
+    fwd = 6.0 * d * ch + 2.0 * T * d * N
+    bwd = 12.0 * d * ch + 4.0 * T * d * N
+    return fwd, bwd, ch
+
+
+def stage_work(counts, cfg):
+    """Algorithmic FLOPs (tensor-bound stages) or bytes (HBM-bound stages) per step, per stage."""
+    d, T, N, k = cfg.d_model, cfg.n_tokens, cfg.n_experts, cfg.top_k
+    ch = float(sum(int(c) * h for c, h in zip(counts, cfg.ffn_sizes)))
+    R = k * T
+    return [
+        T * d * 2 + T * k * 12,                         # router: read x, write idx/gate/row tables
+        T * k * 16,                                      # rank: integer tables
+        T * d * 2 + R * d * 2,                           # permute: read x once, write k copies
+        4.0 * d * ch,                                    # up/gate GEMM
+        2.0 * d * ch,                                    # down GEMM
+        R * d * 4 + T * d * 2,                           # combine: read fp32 rows, write y
+        T * d * 2 + R * d * 4 + R * d * 2,               # dg + permute of dY
+        2.0 * d * ch,                                    # down dgrad
+        2.0 * d * ch,                                    # down wgrad
+        4.0 * d * ch,                                    # up/gate dgrad
+        4.0 * d * ch,                                    # up/gate wgrad
+        T * d * 2 + R * d * 4 + T * d * 2,               # router backward: read x, dxp, write dx
+    ]
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+                for nme, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nme)
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_oracle_sample(inp, n_tok):
+    """fp64 checker, forward + full backward, on the first n_tok tokens as one batch."""
+    from oracle import modse_oracle as O
+    f = lambda a: np.asarray(a, dtype=np.float64)
+    x, dy = f(inp.x[:n_tok]), f(inp.dy[:n_tok])
+    wr = f(inp.w_router)
+    wg = [f(w) for w in inp.w_gate]; wu = [f(w) for w in inp.w_up]; wd = [f(w) for w in inp.w_down]
+    t0 = time.perf_counter()
+    y, rt = O.forward(x, wr, wg, wu, wd, inp.cfg.top_k)
+    O.backward(x, wr, wg, wu, wd, rt, dy)
+    dt = time.perf_counter() - t0
+    return n_tok / dt, dt, O.num_threads()
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    inp = I.generate(cfg)
+    n_tok = args.cpu_tokens
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        cpu_oracle_sample(inp, n_tok)
+    times, cores = [], 1
+    for _ in range(args.steps):
+        tps, dt, cores = cpu_oracle_sample(inp, n_tok)
+        times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = n_tok / (ms / 1e3)
+    sample = f"first {n_tok} tokens of the workload as one batch, forward + full backward"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "d_model": cfg.d_model, "ffn_sizes": list(cfg.ffn_sizes),
+                   "top_k": cfg.top_k, "n_tokens": cfg.n_tokens, "pass": "fwd+bwd"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="train_16k", choices=sorted(I.CONFIGS))
+    ap.add_argument("--cpu-tokens", type=int, default=48, help="tokens of the CPU baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = I.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2409_12210_b200 import binding as B, build as lib_build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    lib_build.build()
+    dev = torch.device("cuda", local_rank)
+
+    inp = I.generate(cfg)
+    dt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
+    T, d, K, W = cfg.n_tokens, cfg.d_model, args.steps, max(args.warmup, 3)
+    layer = B.ModseLayer(d, cfg.ffn_sizes, cfg.top_k)
+    wr, wg, wu, wd = B.pack_weights(inp, dev)
+    x = torch.from_numpy(inp.x).to(dev, dt)
+    dy = torch.from_numpy(inp.dy).to(dev, dt)
+    y, dx = torch.empty_like(x), torch.empty_like(x)
+    dwr = torch.empty(wr.shape, dtype=torch.float32, device=dev)
+    dwg, dwu, dwd = torch.empty_like(wg), torch.empty_like(wu), torch.empty_like(wd)
+    do_bwd = cfg.backward
+    ws = layer.alloc_workspace(dt, T, do_bwd, dev)
+
+    def step():
+        layer.forward(wr, wg, wu, wd, x, y, ws, do_bwd)
+        n = layer.last_launch_count()
+        if do_bwd:
+            layer.backward(wr, wg, wu, wd, x, dy, dx, dwr, dwg, dwu, dwd, ws)
+            n += layer.last_launch_count()
+        return n
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(W):
+        launches_per_step = step()
+    torch.cuda.synchronize()
+    status = layer.check_device_status(ws)
+    if status != 0:
+        raise SystemExit(f"device status {status}: {B.status_string(status)}")
+    counts = layer.get_routing(ws, T)["counts"].cpu().numpy()
+
+    # ---- device-resident timing: K steps between two events, stages bracketed by the library's own events ----
+    sampler = ClockSampler(local_rank)
+    n_calls = K * (2 if do_bwd else 1)
+    layer.stage_timing_begin(n_calls)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    sampler.start()
+    ev0.record()
+    for _ in range(K):
+        step()
+    ev1.record()
+    sync_all()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    stage_ms = layer.stage_timing_end(n_calls)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / K
+    value = world * T / (ms_step / 1e3)
+
+    # ---- end to end: pinned host inputs in, results out, every step ----
+    hx, hdy = torch.from_numpy(inp.x).to(dt).pin_memory(), torch.from_numpy(inp.dy).to(dt).pin_memory()
+    hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+    h2d = hx.numel() * hx.element_size() * (2 if do_bwd else 1)
+    d2h = hy.numel() * hy.element_size() * (2 if do_bwd else 1)
+
+    def e2e_step():
+        x.copy_(hx, non_blocking=True)
+        if do_bwd:
+            dy.copy_(hdy, non_blocking=True)
+        step()
+        hy.copy_(y, non_blocking=True)
+        if do_bwd:
+            hdx.copy_(dx, non_blocking=True)
+
+    for _ in range(3):
+        e2e_step()
+    sync_all()
+    ev0.record()
+    for _ in range(K):
+        e2e_step()
+    ev1.record()
+    sync_all()
+    ms_e2e = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms_e2e], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_value = world * T / (ms_e2e / K / 1e3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of every stage, and of the dominant one ----
+    pk, pk_src = peaks()
+    fwd_flops, bwd_flops, _ = expert_flops(counts, cfg)
+    flops_step = fwd_flops + (bwd_flops if do_bwd else 0.0)
+    work = stage_work(counts, cfg)
+    stages = []
+    for i in range(B.N_STAGES):
+        vals = stage_ms[:, i]
+        vals = vals[vals >= 0]
+        if len(vals) == 0:
+            continue
+        ms = float(vals.mean())
+        if STAGE_BOUND[i] == "tensor":
+            ach, peak, unit = work[i] / (ms * 1e-3) / 1e12, pk["bf16_tflops_sustained"], "TFLOP/s"
+        else:
+            ach, peak, unit = work[i] / (ms * 1e-3) / 1e9, pk["hbm_gbs"], "GB/s"
+        stages.append({"stage": B.stage_name(i), "ms": round(ms, 4), "bound": STAGE_BOUND[i],
+                       "achieved": round(ach, 1), "unit": unit, "frac": round(ach / peak, 4)})
+    dom = max(stages, key=lambda s: s["ms"])
+    roofline = {"kernel": dom["stage"], "bound": dom["bound"], "achieved": dom["achieved"],
+                "peak": pk["bf16_tflops_sustained"] if dom["bound"] == "tensor" else pk["hbm_gbs"],
+                "unit": dom["unit"], "frac": dom["frac"], "traffic": None, "peak_source": f"of {pk_src}",
+                "ms_per_launch": dom["ms"]}
+
+    cpu = None
+    if not args.no_cpu_baseline and world == 1:
+        tps, secs, cores = cpu_oracle_sample(inp, args.cpu_tokens)
+        cpu = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": round(secs, 2),
+               "sample": f"first {args.cpu_tokens} tokens of the workload as one batch, forward + full backward"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "d_model": d, "ffn_sizes": list(cfg.ffn_sizes), "top_k": cfg.top_k,
+                   "n_tokens": T, "pass": "fwd+bwd" if do_bwd else "fwd", "parallelism": f"replicas x{world}",
+                   "l2": "inputs larger than L2 (weights 554 MB, activations > 126 MB per step)"},
+        "tflops": flops_step / (ms_step * 1e-3) / 1e12,
+        "tflops_frac_of_sustained_peak": flops_step / (ms_step * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
+        "counts": [int(c) for c in counts],
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": ms_e2e / K},
+        "gpu_launches": int(launches_per_step * K),
+        "roofline": roofline,
+        "stages": stages,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

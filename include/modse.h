@@ -151,6 +151,27 @@ modse_status_t modse_check_device_status(modse_layer_t *layer, const void *works
  * enqueued (for launch accounting in benchmarks).                            */
 int modse_last_launch_count(const modse_layer_t *layer);
 
+/* Output precision of a bf16 layer.  Off (default): y, dx and the expert weight
+ * gradients are bf16 like the inputs.  On: the same fp32 accumulators are
+ * written as fp32 instead ([T,d] y and dx, [S,d]/[d,S] weight gradients of 4
+ * bytes per element), which removes the last bf16 rounding - e.g. for gradient
+ * accumulation over micro-batches in fp32.  No effect on fp32 layers.        */
+modse_status_t modse_set_output_f32(modse_layer_t *layer, int on);
+
+/* Per-stage device timing (profiling aid).  After modse_stage_timing_begin the
+ * next max_calls forward/backward calls on this layer bracket each of their
+ * stages with a pair of CUDA events on the call's stream (no work is skipped
+ * or reordered).  modse_stage_timing_end waits for those events, writes
+ * ms_out[call * MODSE_N_STAGES + stage] (milliseconds; -1 for a stage the call
+ * did not run), the number of calls seen, and switches timing off again.
+ * Stages 0-5 belong to forward (router, rank, permute, up/gate GEMM + SwiGLU,
+ * down GEMM, combine), 6-11 to backward (dg + permute of dY, down dgrad +
+ * SwiGLU backward, down wgrad, up/gate dgrad, up/gate wgrad, router backward). */
+#define MODSE_N_STAGES 12
+modse_status_t modse_stage_timing_begin(modse_layer_t *layer, int max_calls);
+modse_status_t modse_stage_timing_end(modse_layer_t *layer, float *ms_out, int *calls_out);
+const char *modse_stage_name(int stage);
+
 /* Debugging aid, process-wide: when on, bf16 layers run their grouped GEMMs on
  * the fp32-FMA kernels of the fp32 type (with bf16 storage) instead of the
  * tensor-core kernels - slow, meant for cross-checking.  Such a forward must

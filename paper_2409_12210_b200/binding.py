@@ -23,6 +23,7 @@ MODSE_ERR_DEVICE_TIMEOUT = 6
 MODSE_ERR_DEVICE_BOUNDS = 7
 MODSE_F32 = 0
 MODSE_BF16 = 1
+N_STAGES = 12
 
 
 class ModseError(RuntimeError):
@@ -83,6 +84,14 @@ def load():
     lib.modse_check_device_status.argtypes = [vp, vp, vp]
     lib.modse_last_launch_count.restype = ci
     lib.modse_last_launch_count.argtypes = [vp]
+    lib.modse_set_output_f32.restype = ci
+    lib.modse_set_output_f32.argtypes = [vp, ci]
+    lib.modse_stage_timing_begin.restype = ci
+    lib.modse_stage_timing_begin.argtypes = [vp, ci]
+    lib.modse_stage_timing_end.restype = ci
+    lib.modse_stage_timing_end.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ip]
+    lib.modse_stage_name.restype = ctypes.c_char_p
+    lib.modse_stage_name.argtypes = [ci]
     lib.modse_debug_use_fma_path.restype = None
     lib.modse_debug_use_fma_path.argtypes = [ci]
     _lib = lib
@@ -91,6 +100,10 @@ def load():
 
 def status_string(status: int) -> str:
     return load().modse_status_string(int(status)).decode()
+
+
+def stage_name(i: int) -> str:
+    return load().modse_stage_name(int(i)).decode()
 
 
 def debug_use_fma_path(on: bool) -> None:
@@ -206,6 +219,26 @@ class ModseLayer:
 
     def check_device_status(self, workspace) -> int:
         return int(load().modse_check_device_status(self._h, workspace.data_ptr(), self._stream()))
+
+    def set_output_f32(self, on: bool) -> None:
+        st = load().modse_set_output_f32(self._h, int(bool(on)))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_set_output_f32")
+
+    def stage_timing_begin(self, max_calls: int) -> None:
+        st = load().modse_stage_timing_begin(self._h, int(max_calls))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_stage_timing_begin")
+
+    def stage_timing_end(self, max_calls: int):
+        """[calls, N_STAGES] array of stage times in ms (-1: stage not run by that call)."""
+        import numpy as np
+        buf = (ctypes.c_float * (max_calls * N_STAGES))()
+        n = ctypes.c_int(0)
+        st = load().modse_stage_timing_end(self._h, buf, ctypes.byref(n))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_stage_timing_end")
+        return np.ctypeslib.as_array(buf).reshape(max_calls, N_STAGES)[:n.value].copy()
 
     def last_launch_count(self) -> int:
         return int(load().modse_last_launch_count(self._h))

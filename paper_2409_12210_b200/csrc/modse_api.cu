@@ -17,7 +17,12 @@ struct modse_layer {
     int fwd_dtype = -1;
     int fwd_saved = 0;
     int last_launches = 0;
-    modse::TcPlan tc;             // tensor-map cache of the bf16 path
+    int out_f32 = 0;              // bf16 layers: write y, dx and expert weight gradients as fp32
+    modse::TcPlan tc;             // device facts of the bf16 path
+    // optional per-stage device timing: events [call][stage][start/stop]
+    std::vector<cudaEvent_t> ev;
+    std::vector<unsigned char> ev_used;   // [call][stage]
+    int ev_calls_max = 0, ev_calls = 0;
 };
 
 namespace modse {
@@ -172,8 +177,17 @@ modse_layer_t *modse_create(int d_model, int n_experts, const int *ffn_sizes, in
 
 modse_status_t modse_last_create_error(void) { return g_create_error; }
 
+static void drop_events(modse_layer *L)
+{
+    for (cudaEvent_t e : L->ev) cudaEventDestroy(e);
+    L->ev.clear();
+    L->ev_used.clear();
+    L->ev_calls_max = L->ev_calls = 0;
+}
+
 modse_status_t modse_destroy(modse_layer_t *layer)
 {
+    if (layer) drop_events(layer);
     delete layer;
     return MODSE_OK;
 }
@@ -218,6 +232,30 @@ size_t modse_workspace_bytes(const modse_layer_t *layer, modse_dtype_t dtype, in
         if (ce__ != cudaSuccess) return MODSE_ERR_CUDA; \
     } while (0)
 
+// Brackets one stage with a pair of events when stage timing is on.
+struct StageTimer {
+    modse_layer *L;
+    cudaStream_t s;
+    int call;
+    StageTimer(modse_layer *layer, cudaStream_t stream) : L(layer), s(stream), call(-1)
+    {
+        if (L->ev_calls_max > 0 && L->ev_calls < L->ev_calls_max) call = L->ev_calls++;
+    }
+    void mark(int stage, int which)
+    {
+        if (call < 0) return;
+        const size_t i = ((size_t)call * MODSE_N_STAGES + stage);
+        cudaEventRecord(L->ev[i * 2 + which], s);
+        if (which == 1) L->ev_used[i] = 1;
+    }
+};
+#define MODSE_STAGE(timer, stage, expr) \
+    do {                                \
+        (timer).mark((stage), 0);       \
+        MODSE_CUDA(expr);               \
+        (timer).mark((stage), 1);       \
+    } while (0)
+
 static modse_status_t check_common(const modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *w,
                                    int n_tokens, const void *workspace, size_t workspace_bytes, int save)
 {
@@ -248,26 +286,33 @@ modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const mo
     const WsPtrs p = carve(workspace, L);
     int launches = 0;
     layer->fwd_ws = nullptr;
+    const bool of32 = dtype == MODSE_BF16 && layer->out_f32 != 0;
+    if (of32 && tc_force_simt()) return MODSE_ERR_UNSUPPORTED;
 
+    StageTimer tm(layer, s);
     MODSE_CUDA(cudaMemsetAsync(p.status, 0, 64, s));
-    MODSE_CUDA(launch_router(dtype, m, x, weights->w_router, n_tokens, p, s, &launches));
-    MODSE_CUDA(launch_rank(m, n_tokens, L.Pmax, p, s, &launches));
-    MODSE_CUDA(launch_permute(dtype, m, x, n_tokens, p, s, &launches));
+    MODSE_STAGE(tm, 0, launch_router(dtype, m, x, weights->w_router, n_tokens, p, s, &launches));
+    MODSE_STAGE(tm, 1, launch_rank(m, n_tokens, L.Pmax, p, s, &launches));
+    MODSE_STAGE(tm, 2, launch_permute(dtype, m, x, n_tokens, p, s, &launches));
     if (dtype == MODSE_F32 || tc_force_simt()) {
         // the bf16 cross-check path materialises both pre-activations, which only a saved forward has room for
         if (dtype == MODSE_BF16 && !save) return MODSE_ERR_UNSUPPORTED;
         SimtGemmArgs a{p.xp, weights->w_gate, p.a_pre, 0};
+        tm.mark(3, 0);
         MODSE_CUDA(launch_simt_gemm(dtype, kUpGate, m, L.Pmax, p, a, s, &launches));
         a.wgt = weights->w_up; a.out = p.b_pre;
         MODSE_CUDA(launch_simt_gemm(dtype, kUpGate, m, L.Pmax, p, a, s, &launches));
         MODSE_CUDA(launch_swiglu_fwd(dtype, m, p, L.hb, s, &launches));
+        tm.mark(3, 1);
         SimtGemmArgs b{p.hm, weights->w_down, p.o, 0};
-        MODSE_CUDA(launch_simt_gemm(dtype, kDown, m, L.Pmax, p, b, s, &launches));
+        MODSE_STAGE(tm, 4, launch_simt_gemm(dtype, kDown, m, L.Pmax, p, b, s, &launches));
     } else {
-        st = tc_forward(layer->tc, m, L, p, weights, save, s, &launches);
-        if (st != MODSE_OK) return st;
+        TcMaps maps;
+        if (!tc_fill_maps(maps, m, L, p, weights, false)) return MODSE_ERR_CUDA;
+        MODSE_STAGE(tm, 3, tc_launch(layer->tc, TcUpGate, maps, m, p, nullptr, save, false, s, &launches));
+        MODSE_STAGE(tm, 4, tc_launch(layer->tc, TcDown, maps, m, p, nullptr, save, false, s, &launches));
     }
-    MODSE_CUDA(launch_combine(dtype, m, n_tokens, p, y, s, &launches));
+    MODSE_STAGE(tm, 5, launch_combine(dtype, m, n_tokens, p, y, of32, s, &launches));
 
     layer->fwd_ws = workspace;
     layer->fwd_tokens = n_tokens;
@@ -296,28 +341,41 @@ modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const m
     const WsLayout L = make_layout(m, layer->h_desc.data(), dtype == MODSE_F32 ? 4 : 2, n_tokens, true);
     const WsPtrs p = carve(workspace, L);
     int launches = 0;
+    const bool of32 = dtype == MODSE_BF16 && layer->out_f32 != 0;
+    if (of32 && tc_force_simt()) return MODSE_ERR_UNSUPPORTED;
 
-    MODSE_CUDA(launch_dg_permute(dtype, m, dy, n_tokens, p, s, &launches));
+    StageTimer tm(layer, s);
+    MODSE_STAGE(tm, 6, launch_dg_permute(dtype, m, dy, n_tokens, p, s, &launches));
     if (dtype == MODSE_F32 || tc_force_simt()) {
         SimtGemmArgs a{p.dyp, weights->w_down, p.da, 0};                       // dHm into the dA buffer
+        tm.mark(7, 0);
         MODSE_CUDA(launch_simt_gemm(dtype, kDownDgrad, m, L.Pmax, p, a, s, &launches));
         MODSE_CUDA(launch_swiglu_bwd(dtype, m, p, L.hb, s, &launches));
+        tm.mark(7, 1);
         SimtGemmArgs w{p.dyp, p.hm, wgrads->dw_down, 0};
-        MODSE_CUDA(launch_simt_gemm(dtype, kDownWgrad, m, L.Pmax, p, w, s, &launches));
+        MODSE_STAGE(tm, 8, launch_simt_gemm(dtype, kDownWgrad, m, L.Pmax, p, w, s, &launches));
         SimtGemmArgs g{p.da, weights->w_gate, p.dxp, 0};
+        tm.mark(9, 0);
         MODSE_CUDA(launch_simt_gemm(dtype, kUpGateDgrad, m, L.Pmax, p, g, s, &launches));
         g.act = p.db; g.wgt = weights->w_up; g.accumulate = 1;
         MODSE_CUDA(launch_simt_gemm(dtype, kUpGateDgrad, m, L.Pmax, p, g, s, &launches));
+        tm.mark(9, 1);
         SimtGemmArgs wg{p.da, p.xp, wgrads->dw_gate, 0};
+        tm.mark(10, 0);
         MODSE_CUDA(launch_simt_gemm(dtype, kUpGateWgrad, m, L.Pmax, p, wg, s, &launches));
         wg.act = p.db; wg.out = wgrads->dw_up;
         MODSE_CUDA(launch_simt_gemm(dtype, kUpGateWgrad, m, L.Pmax, p, wg, s, &launches));
+        tm.mark(10, 1);
     } else {
-        st = tc_backward(layer->tc, m, L, p, weights, wgrads, s, &launches);
-        if (st != MODSE_OK) return st;
+        TcMaps maps;
+        if (!tc_fill_maps(maps, m, L, p, weights, true)) return MODSE_ERR_CUDA;
+        MODSE_STAGE(tm, 7, tc_launch(layer->tc, TcDownDgrad, maps, m, p, wgrads, true, of32, s, &launches));
+        MODSE_STAGE(tm, 8, tc_launch(layer->tc, TcDownWgrad, maps, m, p, wgrads, true, of32, s, &launches));
+        MODSE_STAGE(tm, 9, tc_launch(layer->tc, TcUpGateDgrad, maps, m, p, wgrads, true, of32, s, &launches));
+        MODSE_STAGE(tm, 10, tc_launch(layer->tc, TcUpGateWgrad, maps, m, p, wgrads, true, of32, s, &launches));
     }
-    MODSE_CUDA(launch_router_bwd(dtype, m, x, weights->w_router, n_tokens, L.nblk_bwd, p, dx,
-                                 static_cast<float *>(wgrads->dw_router), s, &launches));
+    MODSE_STAGE(tm, 11, launch_router_bwd(dtype, m, x, weights->w_router, n_tokens, L.nblk_bwd, p, dx, of32,
+                                          static_cast<float *>(wgrads->dw_router), s, &launches));
     layer->last_launches = launches;
     return MODSE_OK;
 }
@@ -370,6 +428,64 @@ modse_status_t modse_check_device_status(modse_layer_t *layer, const void *works
 
 int modse_last_launch_count(const modse_layer_t *layer) { return layer ? layer->last_launches : 0; }
 
+modse_status_t modse_set_output_f32(modse_layer_t *layer, int on)
+{
+    if (layer == nullptr) return MODSE_ERR_INVALID_ARG;
+    layer->out_f32 = on ? 1 : 0;
+    return MODSE_OK;
+}
+
 void modse_debug_use_fma_path(int on) { tc_set_force_simt(on); }
+
+const char *modse_stage_name(int stage)
+{
+    static const char *names[MODSE_N_STAGES] = {"router", "rank", "permute", "upgate_gemm_swiglu", "down_gemm",
+                                                "combine", "dg_permute", "down_dgrad_swiglu_bwd", "down_wgrad",
+                                                "upgate_dgrad", "upgate_wgrad", "router_bwd"};
+    return (stage >= 0 && stage < MODSE_N_STAGES) ? names[stage] : "";
+}
+
+modse_status_t modse_stage_timing_begin(modse_layer_t *layer, int max_calls)
+{
+    if (layer == nullptr || max_calls < 1 || max_calls > 4096) return MODSE_ERR_INVALID_ARG;
+    drop_events(layer);
+    const size_t n = (size_t)max_calls * MODSE_N_STAGES * 2;
+    layer->ev.reserve(n);
+    for (size_t i = 0; i < n; ++i) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) {
+            drop_events(layer);
+            return MODSE_ERR_CUDA;
+        }
+        layer->ev.push_back(e);
+    }
+    layer->ev_used.assign((size_t)max_calls * MODSE_N_STAGES, 0);
+    layer->ev_calls_max = max_calls;
+    layer->ev_calls = 0;
+    return MODSE_OK;
+}
+
+modse_status_t modse_stage_timing_end(modse_layer_t *layer, float *ms_out, int *calls_out)
+{
+    if (layer == nullptr || ms_out == nullptr || calls_out == nullptr) return MODSE_ERR_INVALID_ARG;
+    const int calls = layer->ev_calls;
+    modse_status_t st = MODSE_OK;
+    for (int c = 0; c < calls; ++c)
+        for (int sidx = 0; sidx < MODSE_N_STAGES; ++sidx) {
+            const size_t i = (size_t)c * MODSE_N_STAGES + sidx;
+            float ms = -1.0f;
+            if (layer->ev_used[i]) {
+                if (cudaEventSynchronize(layer->ev[i * 2 + 1]) != cudaSuccess ||
+                    cudaEventElapsedTime(&ms, layer->ev[i * 2], layer->ev[i * 2 + 1]) != cudaSuccess) {
+                    st = MODSE_ERR_CUDA;
+                    ms = -1.0f;
+                }
+            }
+            ms_out[i] = ms;
+        }
+    *calls_out = calls;
+    drop_events(layer);
+    return st;
+}
 
 }  // extern "C"

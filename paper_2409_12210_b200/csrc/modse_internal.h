@@ -57,13 +57,13 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
 cudaError_t launch_rank(const LayerMeta &m, int T, int Pmax, const WsPtrs &p, cudaStream_t s, int *launches);
 cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, const WsPtrs &p,
                            cudaStream_t s, int *launches);
-cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, cudaStream_t s,
-                           int *launches);
+cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, bool out_f32,
+                           cudaStream_t s, int *launches);
 cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, const WsPtrs &p,
                               cudaStream_t s, int *launches);
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
-                              int nblk_bwd, const WsPtrs &p, void *dx, float *dw_router, cudaStream_t s,
-                              int *launches);
+                              int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
+                              cudaStream_t s, int *launches);
 
 // ---- fp32-FMA grouped GEMMs and SwiGLU elementwise (simt_gemm.cu) ----
 enum GemmKind : int {

@@ -307,10 +307,10 @@ permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int
 // ---------------------------------------------------------------------------
 // Combine (Eq. 4): y_t = g[t,0]*o[row(t,0)] + g[t,1]*o[row(t,1)], fp32, slot order.
 // ---------------------------------------------------------------------------
-template <typename T>
+template <typename TO>
 __global__ void __launch_bounds__(256)
 combine_kernel(const float *__restrict__ o, int Ttok, int d, int k, const int *__restrict__ prow_of,
-               const float *__restrict__ topk_gate, T *__restrict__ y)
+               const float *__restrict__ topk_gate, TO *__restrict__ y)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * 8 + warp;
@@ -380,13 +380,13 @@ dg_permute_kernel(const T *__restrict__ dy, const float *__restrict__ o, int Tto
 // Phase B (thread per column): partial dW_router over this block's tokens in
 // ascending token order, kept in shared memory [N][dc] and written out.
 // ---------------------------------------------------------------------------
-template <typename T>
+template <typename T, typename TO>
 __global__ void __launch_bounds__(256)
 router_bwd_kernel(const T *__restrict__ x, const T *__restrict__ w_router, const float *__restrict__ dxp,
                   int Ttok,
                   int d, int N, int k, int dc, const int *__restrict__ topk_idx,
                   const float *__restrict__ topk_gate, const int *__restrict__ prow_of,
-                  const float *__restrict__ dg, float *__restrict__ dz, T *__restrict__ dx,
+                  const float *__restrict__ dg, float *__restrict__ dz, TO *__restrict__ dx,
                   float *__restrict__ dwr_partial)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -535,11 +535,11 @@ cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, 
     return cudaSuccess;
 }
 
-cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, cudaStream_t s,
-                           int *launches)
+cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, bool out_f32,
+                           cudaStream_t s, int *launches)
 {
     const int grid = (T + 7) / 8;
-    if (dt == MODSE_F32)
+    if (dt == MODSE_F32 || out_f32)
         combine_kernel<float><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of, p.topk_gate,
                                                    (float *)y);
     else
@@ -567,9 +567,21 @@ cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *
     return cudaSuccess;
 }
 
+template <typename T, typename TO>
+static cudaError_t run_router_bwd(dim3 grid, size_t smem, cudaStream_t s, const LayerMeta &m, const void *x,
+                                  const void *w_router, int T_tok, int dc, const WsPtrs &p, void *dx)
+{
+    auto kern = router_bwd_kernel<T, TO>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, 256, smem, s>>>((const T *)x, (const T *)w_router, (const float *)p.dxp, T_tok, m.d, m.N, m.k, dc,
+                                 p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz, (TO *)dx, p.dwr_partial);
+    return cudaSuccess;
+}
+
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
-                              int nblk_bwd, const WsPtrs &p, void *dx, float *dw_router, cudaStream_t s,
-                              int *launches)
+                              int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
+                              cudaStream_t s, int *launches)
 {
     // column chunk so that the [N][dc] fp32 accumulator fits in 64 KB of shared memory
     int dc = m.d;
@@ -578,21 +590,11 @@ cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *
     const size_t smem =
         sizeof(float) * kRouterBwdTokB * 2 + sizeof(int) * kRouterBwdTokB * 2 + sizeof(float) * m.N * dc;
     dim3 grid(nblk_bwd, ychunks);
-    if (dt == MODSE_F32) {
-        auto kern = router_bwd_kernel<float>;
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        kern<<<grid, 256, smem, s>>>((const float *)x, (const float *)w_router, (const float *)p.dxp, T, m.d, m.N,
-                                     m.k, dc, p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz, (float *)dx,
-                                     p.dwr_partial);
-    } else {
-        auto kern = router_bwd_kernel<__nv_bfloat16>;
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        kern<<<grid, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router,
-                                     (const float *)p.dxp, T, m.d, m.N, m.k, dc, p.topk_idx, p.topk_gate,
-                                     p.prow_of, p.dg, p.dz, (__nv_bfloat16 *)dx, p.dwr_partial);
-    }
+    cudaError_t re;
+    if (dt == MODSE_F32) re = run_router_bwd<float, float>(grid, smem, s, m, x, w_router, T, dc, p, dx);
+    else if (out_f32) re = run_router_bwd<__nv_bfloat16, float>(grid, smem, s, m, x, w_router, T, dc, p, dx);
+    else re = run_router_bwd<__nv_bfloat16, __nv_bfloat16>(grid, smem, s, m, x, w_router, T, dc, p, dx);
+    if (re != cudaSuccess) return re;
     MODSE_LAUNCH_CHECK();
     const int n = m.N * m.d;
     reduce_dwr_kernel<<<(n + 255) / 256, 256, 0, s>>>(p.dwr_partial, nblk_bwd, n, dw_router);

@@ -44,8 +44,6 @@ void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
 
 namespace {
 
-enum TcKind : int { TcUpGate = 0, TcDown = 1, TcDownDgrad = 2, TcDownWgrad = 3, TcUpGateDgrad = 4, TcUpGateWgrad = 5 };
-
 constexpr int kStages = 4;
 constexpr int kBoxBytes = 64 * 64 * 2;           // one TMA box: 64 rows of 128 bytes
 constexpr int kARegion = 2 * kBoxBytes;          // 128 rows (or 128 MN elements) x 64 K
@@ -56,10 +54,6 @@ constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 
-struct TcMaps {
-    CUtensorMap xp, dyp, wgate, wup, wdown, hm, da, db;
-};
-
 struct TcParams {
     LayerMeta meta;
     const int *poffsets;
@@ -69,6 +63,7 @@ struct TcParams {
     float *o, *dxp;
     __nv_bfloat16 *dw_gate, *dw_up, *dw_down;
     int save;
+    int out_f32;   // weight gradients are written as fp32 instead of bf16
 };
 
 // dynamic shared memory map (after 1024-byte alignment)
@@ -391,7 +386,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             store_bf16x32(prm.db + idx, db);
         }
     } else if constexpr (KIND == TcDownWgrad) {
-        __nv_bfloat16 *out = prm.dw_down + (size_t)(t.m0 + row) * S + t.ho + t.n0;
+        const size_t oidx = (size_t)(t.m0 + row) * S + t.ho + t.n0;
         for (int c = 0; c < t.ncols; c += 32) {
             float v[32];
             if (have_acc) {
@@ -404,10 +399,12 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
             }
-            store_bf16x32(out + c, v);
+            if (prm.out_f32) store_f32x32(reinterpret_cast<float *>(prm.dw_down) + oidx + c, v);
+            else store_bf16x32(prm.dw_down + oidx + c, v);
         }
     } else {
-        __nv_bfloat16 *out = (t.which ? prm.dw_up : prm.dw_gate) + (size_t)(t.ho + t.m0 + row) * d + t.n0;
+        __nv_bfloat16 *obase = t.which ? prm.dw_up : prm.dw_gate;
+        const size_t oidx = (size_t)(t.ho + t.m0 + row) * d + t.n0;
         for (int c = 0; c < t.ncols; c += 32) {
             float v[32];
             if (have_acc) {
@@ -420,7 +417,10 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
             }
-            if (row < t.mrows) store_bf16x32(out + c, v);
+            if (row < t.mrows) {
+                if (prm.out_f32) store_f32x32(reinterpret_cast<float *>(obase) + oidx + c, v);
+                else store_bf16x32(obase + oidx + c, v);
+            }
         }
     }
 }
@@ -620,8 +620,10 @@ bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols)
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
-               bool backward)
+}  // namespace
+
+bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
+                  bool backward)
 {
     const uint64_t panel_rows = L.hb / 64;
     bool ok = true;
@@ -642,7 +644,9 @@ bool fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs
     return ok;
 }
 
-TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *g, bool save)
+namespace {
+
+TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *g, bool save, bool out_f32)
 {
     TcParams prm{};
     prm.meta = m;
@@ -662,6 +666,7 @@ TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *
         prm.dw_down = (__nv_bfloat16 *)g->dw_down;
     }
     prm.save = save ? 1 : 0;
+    prm.out_f32 = out_f32 ? 1 : 0;
     return prm;
 }
 
@@ -692,30 +697,20 @@ int sm_count(TcPlan &plan)
 
 }  // namespace
 
-modse_status_t tc_forward(TcPlan &plan, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
-                          const modse_weights_t *w, bool save, cudaStream_t s, int *launches)
+cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const LayerMeta &m, const WsPtrs &p,
+                      const modse_wgrads_t *g, bool save, bool out_f32, cudaStream_t s, int *launches)
 {
-    TcMaps maps;
-    if (!fill_maps(maps, m, L, p, w, false)) return MODSE_ERR_CUDA;
-    const TcParams prm = make_params(m, p, nullptr, save);
+    const TcParams prm = make_params(m, p, g, save, out_f32);
     const int grid = sm_count(plan);
-    if (launch_kind<TcUpGate>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
-    if (launch_kind<TcDown>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
-    return MODSE_OK;
-}
-
-modse_status_t tc_backward(TcPlan &plan, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
-                           const modse_weights_t *w, const modse_wgrads_t *g, cudaStream_t s, int *launches)
-{
-    TcMaps maps;
-    if (!fill_maps(maps, m, L, p, w, true)) return MODSE_ERR_CUDA;
-    const TcParams prm = make_params(m, p, g, true);
-    const int grid = sm_count(plan);
-    if (launch_kind<TcDownDgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
-    if (launch_kind<TcDownWgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
-    if (launch_kind<TcUpGateDgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
-    if (launch_kind<TcUpGateWgrad>(maps, prm, grid, s, launches) != cudaSuccess) return MODSE_ERR_CUDA;
-    return MODSE_OK;
+    switch (kind) {
+    case TcUpGate: return launch_kind<TcUpGate>(maps, prm, grid, s, launches);
+    case TcDown: return launch_kind<TcDown>(maps, prm, grid, s, launches);
+    case TcDownDgrad: return launch_kind<TcDownDgrad>(maps, prm, grid, s, launches);
+    case TcDownWgrad: return launch_kind<TcDownWgrad>(maps, prm, grid, s, launches);
+    case TcUpGateDgrad: return launch_kind<TcUpGateDgrad>(maps, prm, grid, s, launches);
+    case TcUpGateWgrad: return launch_kind<TcUpGateWgrad>(maps, prm, grid, s, launches);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace modse

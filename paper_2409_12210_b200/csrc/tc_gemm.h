@@ -1,6 +1,8 @@
 // Tensor-core (tcgen05 / TMEM / TMA) grouped GEMM stages of the bf16 layer.
 #pragma once
 
+#include <cuda.h>
+
 #include "modse_internal.h"
 
 namespace modse {
@@ -15,13 +17,24 @@ struct TcPlan {
 bool tc_force_simt();
 void tc_set_force_simt(int on);
 
-// Grouped up/gate projection with fused SwiGLU, then grouped down projection
-// into the fp32 buffer o (Sec. 3.1, Eq. 4, expert by expert).
-modse_status_t tc_forward(TcPlan &plan, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
-                          const modse_weights_t *w, bool save, cudaStream_t s, int *launches);
-// Down-projection dgrad with fused SwiGLU backward, down wgrad, up/gate dgrad
-// into the fp32 buffer dxp, up/gate wgrads.
-modse_status_t tc_backward(TcPlan &plan, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
-                           const modse_weights_t *w, const modse_wgrads_t *g, cudaStream_t s, int *launches);
+// The six grouped products of the layer (Sec. 3.1, Eq. 4 and its gradient).
+enum TcKind : int {
+    TcUpGate = 0,       // Hm = silu(xp Wg^T) * (xp Wu^T), optionally saving both pre-activations
+    TcDown = 1,         // o = Hm Wd^T into the fp32 buffer o
+    TcDownDgrad = 2,    // dHm = dyp Wd, fused SwiGLU backward -> dA, dB
+    TcDownWgrad = 3,    // dWd = dyp^T Hm
+    TcUpGateDgrad = 4,  // dxp = dA Wg + dB Wu into the fp32 buffer dxp
+    TcUpGateWgrad = 5   // dWg = dA^T xp, dWu = dB^T xp
+};
+
+// Tensor maps of every TMA-loaded buffer (bf16, 64 x 64 boxes, 128-byte swizzle).
+struct TcMaps {
+    CUtensorMap xp, dyp, wgate, wup, wdown, hm, da, db;
+};
+
+bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
+                  bool backward);
+cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const LayerMeta &m, const WsPtrs &p,
+                      const modse_wgrads_t *g, bool save, bool out_f32, cudaStream_t s, int *launches);
 
 }  // namespace modse

@@ -40,7 +40,15 @@ def rel_err_beyond_storage(got, ref) -> float:
     return float(excess.max() / rms) if rms > 0 else float(excess.max())
 
 
-def run_gpu(inp: I.LayerInputs, backward: bool, save: bool | None = None):
+def rms_rel_err(got, ref) -> float:
+    """RMS(got - ref) / RMS(ref)."""
+    got = np.asarray(got, dtype=np.float64); ref = np.asarray(ref, dtype=np.float64)
+    rms = float(np.sqrt(np.mean(ref ** 2))) if ref.size else 0.0
+    err = float(np.sqrt(np.mean((got - ref) ** 2))) if ref.size else 0.0
+    return err / rms if rms > 0 else err
+
+
+def run_gpu(inp: I.LayerInputs, backward: bool, save: bool | None = None, out_f32: bool = False):
     """Forward (and backward) through the C ABI; returns host numpy results."""
     import torch
     from paper_2409_12210_b200 import binding as B
@@ -48,10 +56,12 @@ def run_gpu(inp: I.LayerInputs, backward: bool, save: bool | None = None):
     dt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
     dev = "cuda"
     layer = B.ModseLayer(cfg.d_model, cfg.ffn_sizes, cfg.top_k)
+    layer.set_output_f32(out_f32)
+    odt = torch.float32 if out_f32 else dt
     wr, wg, wu, wd = B.pack_weights(inp, dev)
     x = torch.from_numpy(inp.x).to(dev, dt)
     T = x.shape[0]
-    y = torch.empty_like(x)
+    y = torch.empty(x.shape, dtype=odt, device=dev)
     save = backward if save is None else save
     ws = layer.alloc_workspace(dt, T, save)
     layer.forward(wr, wg, wu, wd, x, y, ws, save)
@@ -62,9 +72,9 @@ def run_gpu(inp: I.LayerInputs, backward: bool, save: bool | None = None):
     out["routing"] = {k: v.cpu().numpy().copy() for k, v in rt.items()}
     if backward:
         dy = torch.from_numpy(inp.dy).to(dev, dt)
-        dx = torch.empty_like(x)
+        dx = torch.empty(x.shape, dtype=odt, device=dev)
         dwr = torch.empty(wr.shape, dtype=torch.float32, device=dev)
-        dwg, dwu, dwd = torch.empty_like(wg), torch.empty_like(wu), torch.empty_like(wd)
+        dwg, dwu, dwd = (torch.empty(w.shape, dtype=odt, device=dev) for w in (wg, wu, wd))
         layer.backward(wr, wg, wu, wd, x, dy, dx, dwr, dwg, dwu, dwd, ws)
         out["launches_bwd"] = layer.last_launch_count()
         dg, dz = layer.get_gate_grads(ws, T)
@@ -93,10 +103,29 @@ def check_routing(gpu_rt, rt, gate_tol=1e-6):
     assert np.max(np.abs(gpu_rt["topk_gate"] - rt.topk_gate)) <= gate_tol
 
 
-def check_all(inp, gpu, ora, tol, discount_storage_rounding=False):
-    """Element-by-element comparison of every output; returns the error table.
-    With discount_storage_rounding the bf16-stored tensors are measured with
-    rel_err_beyond_storage (degenerate shapes only)."""
+def reference_tensors(ora):
+    """Oracle results in the library's layouts, keyed like run_gpu's output."""
+    ref = {"y": ora["y"]}
+    if "g" in ora:
+        g, rt = ora["g"], ora["rt"]
+        ref.update(dx=g.dx, dw_router=g.dw_router, dw_gate=np.concatenate(g.dw_gate, 0),
+                   dw_up=np.concatenate(g.dw_up, 0), dw_down=np.concatenate(g.dw_down, 1), dg=g.dg,
+                   dz=np.take_along_axis(g.dz, rt.topk_idx.astype(np.int64), 1))
+    return ref
+
+
+def check_rms(gpu, ora, tol):
+    """RMS error of every tensor relative to the tensor's RMS (the typical, not the worst, element)."""
+    errs = {k: rms_rel_err(gpu[k], v) for k, v in reference_tensors(ora).items() if k in gpu}
+    bad = {k: v for k, v in errs.items() if not (v <= tol)}
+    assert not bad, f"RMS error over {tol}: {bad} (all: {errs})"
+    return errs
+
+
+def check_all(inp, gpu, ora, tol, discount_storage_rounding=False, only=None):
+    """Element-by-element comparison of every output (or of those named in `only`);
+    returns the error table.  With discount_storage_rounding the tensors stored in
+    bf16 are measured with rel_err_beyond_storage."""
     check_routing(gpu["routing"], ora["rt"])
     full = rel_err
     rel_err_ = rel_err_beyond_storage if discount_storage_rounding else rel_err
@@ -113,6 +142,8 @@ def check_all(inp, gpu, ora, tol, discount_storage_rounding=False):
         dz_kept = np.take_along_axis(g.dz, rt.topk_idx.astype(np.int64), 1)
         errs["dz"] = full(gpu["dz"], dz_kept)
     assert gpu["status"] == 0
+    if only is not None:
+        errs = {k: v for k, v in errs.items() if k in only}
     bad = {k: v for k, v in errs.items() if not (v <= tol)}
     assert not bad, f"over tolerance {tol}: {bad} (all: {errs})"
     return errs
