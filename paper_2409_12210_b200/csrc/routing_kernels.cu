@@ -7,11 +7,11 @@
 //   rank_kernel        exclusive scans of the histogram -> counts, offsets and
 //                      the stable destination row of every (token, slot).
 //   permute_kernel     gathers token rows into padded expert groups.
-//   combine_kernel     y_t = sum_j g[t,j] * o[row(t,j)]  (Sec. 3.1, Eq. 4).
+//   combine_kernel     y_t = sum_j o[row(t,j)], o = gated expert output (Sec. 3.1, Eq. 4).
 //                      (o and dxp, the two buffers that are summed over a
 //                      token's slots, are kept in fp32 for every layer type so
 //                      that the sum is rounded to the layer type only once.)
-//   dg_permute_kernel  dg[t,j] = <dY_t, o_(t,j)>, rows g*dY_t in group order.
+//   dg_permute_kernel  dg[t,j] = <dY_t, E_(t,j)>, rows of dY in group order.
 //   router_bwd_kernel  softmax Jacobian on the kept logits, dx assembly and
 //                      per-block partial sums of dW_router; reduced in block
 //                      order by reduce_dwr_kernel so the result is reproducible.
@@ -305,36 +305,36 @@ permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int
 }
 
 // ---------------------------------------------------------------------------
-// Combine (Eq. 4): y_t = g[t,0]*o[row(t,0)] + g[t,1]*o[row(t,1)], fp32, slot order.
+// Combine (Eq. 4): the gate of each assignment was applied to its hidden row
+// before the down projection (the projection is linear, so g*(W h) = W (g*h)),
+// so y_t = o[row(t,0)] + o[row(t,1)], added in fp32 in slot order.
 // ---------------------------------------------------------------------------
 template <typename TO>
 __global__ void __launch_bounds__(256)
 combine_kernel(const float *__restrict__ o, int Ttok, int d, int k, const int *__restrict__ prow_of,
-               const float *__restrict__ topk_gate, TO *__restrict__ y)
+               TO *__restrict__ y)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * 8 + warp;
     if (t >= Ttok) return;
     const int r0 = prow_of[(size_t)t * k];
-    const float g0 = topk_gate[(size_t)t * k];
     const int r1 = (k > 1) ? prow_of[(size_t)t * k + 1] : -1;
-    const float g1 = (k > 1) ? topk_gate[(size_t)t * k + 1] : 0.f;
     for (int c = lane * 8; c < d; c += 256) {
         float a[8], acc[8];
-        load8(o + (size_t)r0 * d + c, a);
-#pragma unroll
-        for (int u = 0; u < 8; ++u) acc[u] = g0 * a[u];
+        load8(o + (size_t)r0 * d + c, acc);
         if (r1 >= 0) {
             load8(o + (size_t)r1 * d + c, a);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) acc[u] = fmaf(g1, a[u], acc[u]);
+            for (int u = 0; u < 8; ++u) acc[u] += a[u];
         }
         store8(y + (size_t)t * d + c, acc);
     }
 }
 
 // ---------------------------------------------------------------------------
-// Backward entry: dg[t,j] = <dY_t, o_(t,j)>; dyp[row(t,j)] = g[t,j]*dY_t.
+// Backward entry: dg[t,j] = <dY_t, E_(t,j)> = <dY_t, o[row(t,j)]> / g[t,j] (o holds
+// the gated expert output; a gate that underflowed to 0 gives dg = 0, and its
+// dz = g*(dg - s) is 0 either way); dyp[row(t,j)] = dY_t, an exact copy.
 // ---------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
@@ -353,15 +353,15 @@ dg_permute_kernel(const T *__restrict__ dy, const float *__restrict__ o, int Tto
             const float g = topk_gate[(size_t)t * k + j];
             float acc = 0.f;
             for (int c = lane * 8; c < d; c += 256) {
-                float v[8], ov[8], sv[8];
+                float v[8], ov[8];
                 load8(src + c, v);
                 load8(o + (size_t)row * d + c, ov);
 #pragma unroll
-                for (int u = 0; u < 8; ++u) { acc = fmaf(v[u], ov[u], acc); sv[u] = g * v[u]; }
-                store8(dyp + (size_t)row * d + c, sv);
+                for (int u = 0; u < 8; ++u) acc = fmaf(v[u], ov[u], acc);
+                store8(dyp + (size_t)row * d + c, v);
             }
             acc = warp_sum(acc);
-            if (lane == 0) dg[(size_t)t * k + j] = acc;
+            if (lane == 0) dg[(size_t)t * k + j] = (g > 0.f) ? acc / g : 0.f;
         }
     } else {
         const int pb = blockIdx.x - tok_blocks;
@@ -540,11 +540,10 @@ cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const Ws
 {
     const int grid = (T + 7) / 8;
     if (dt == MODSE_F32 || out_f32)
-        combine_kernel<float><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of, p.topk_gate,
-                                                   (float *)y);
+        combine_kernel<float><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of, (float *)y);
     else
         combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of,
-                                                           p.topk_gate, (__nv_bfloat16 *)y);
+                                                           (__nv_bfloat16 *)y);
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
 }

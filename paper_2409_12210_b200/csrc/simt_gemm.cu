@@ -147,32 +147,44 @@ simt_grouped_gemm(int kind, LayerMeta m, const int *__restrict__ poffsets, const
     }
 }
 
-// hm = silu(a) * b over the whole used part of the [rows, h_e] buffers.
+// hm[r,:] = g_r * silu(a[r,:]) * b[r,:] for every padded row r of every expert
+// (g_r = gate of the assignment in that row, 0 for padding rows).
 template <typename T>
 __global__ void __launch_bounds__(256)
-swiglu_fwd_kernel(const T *__restrict__ a, const T *__restrict__ b, T *__restrict__ hm,
-                  const long long *__restrict__ ebase, int N)
+swiglu_fwd_kernel(const T *__restrict__ a, const T *__restrict__ b, T *__restrict__ hm, LayerMeta m,
+                  const int *__restrict__ poffsets, const long long *__restrict__ ebase,
+                  const float *__restrict__ pgate)
 {
-    const long long n = ebase[N];
+    const int e = blockIdx.y;
+    const int he = m.hoff[e + 1] - m.hoff[e];
+    const int cp = poffsets[e + 1] - poffsets[e];
+    const long long n = (long long)cp * he, eb = ebase[e];
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
-        const float av = ld(a, i), bv = ld(b, i);
+        const float g = pgate[poffsets[e] + (int)(i / he)];
+        const float av = ld(a, eb + i), bv = ld(b, eb + i);
         const float sg = 1.0f / (1.0f + expf(-av));
-        st(hm, i, av * sg * bv);
+        st(hm, eb + i, g * (av * sg * bv));
     }
 }
 
-// da = dhm * b * silu'(a), db = dhm * silu(a); dhm arrives in the da buffer.
+// dhm = g_r * (dY W_down) arrives ungated in the da buffer;
+// da = dhm * b * silu'(a), db = dhm * silu(a).
 template <typename T>
 __global__ void __launch_bounds__(256)
 swiglu_bwd_kernel(const T *__restrict__ a, const T *__restrict__ b, T *__restrict__ da, T *__restrict__ db,
-                  const long long *__restrict__ ebase, int N)
+                  LayerMeta m, const int *__restrict__ poffsets, const long long *__restrict__ ebase,
+                  const float *__restrict__ pgate)
 {
-    const long long n = ebase[N];
+    const int e = blockIdx.y;
+    const int he = m.hoff[e + 1] - m.hoff[e];
+    const int cp = poffsets[e + 1] - poffsets[e];
+    const long long n = (long long)cp * he, eb = ebase[e];
     for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) {
-        const float av = ld(a, i), bv = ld(b, i), dh = ld(da, i);
+        const float g = pgate[poffsets[e] + (int)(i / he)];
+        const float av = ld(a, eb + i), bv = ld(b, eb + i), dh = g * ld(da, eb + i);
         const float sg = 1.0f / (1.0f + expf(-av));
-        st(da, i, dh * bv * sg * (1.0f + av * (1.0f - sg)));
-        st(db, i, dh * av * sg);
+        st(da, eb + i, dh * bv * sg * (1.0f + av * (1.0f - sg)));
+        st(db, eb + i, dh * av * sg);
     }
 }
 
@@ -205,25 +217,18 @@ cudaError_t launch_simt_gemm(modse_dtype_t dt, GemmKind kind, const LayerMeta &m
     return cudaSuccess;
 }
 
-static int elementwise_grid(size_t hb)
-{
-    size_t g = (hb + 255) / 256;
-    if (g > 148 * 8) g = 148 * 8;
-    if (g < 1) g = 1;
-    return (int)g;
-}
-
 cudaError_t launch_swiglu_fwd(modse_dtype_t dt, const LayerMeta &m, const WsPtrs &p, size_t hb, cudaStream_t s,
                               int *launches)
 {
-    const int grid = elementwise_grid(hb);
+    (void)hb;
+    dim3 grid(148, m.N);
     if (dt == MODSE_F32)
-        swiglu_fwd_kernel<float><<<grid, 256, 0, s>>>((const float *)p.a_pre, (const float *)p.b_pre, (float *)p.hm,
-                                                      p.ebase, m.N);
+        swiglu_fwd_kernel<float><<<grid, 256, 0, s>>>((const float *)p.a_pre, (const float *)p.b_pre, (float *)p.hm, m,
+                                                      p.poffsets, p.ebase, p.pgate);
     else
         swiglu_fwd_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)p.a_pre,
                                                               (const __nv_bfloat16 *)p.b_pre,
-                                                              (__nv_bfloat16 *)p.hm, p.ebase, m.N);
+                                                              (__nv_bfloat16 *)p.hm, m, p.poffsets, p.ebase, p.pgate);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (launches) ++*launches;
@@ -233,15 +238,16 @@ cudaError_t launch_swiglu_fwd(modse_dtype_t dt, const LayerMeta &m, const WsPtrs
 cudaError_t launch_swiglu_bwd(modse_dtype_t dt, const LayerMeta &m, const WsPtrs &p, size_t hb, cudaStream_t s,
                               int *launches)
 {
-    const int grid = elementwise_grid(hb);
+    (void)hb;
+    dim3 grid(148, m.N);
     if (dt == MODSE_F32)
         swiglu_bwd_kernel<float><<<grid, 256, 0, s>>>((const float *)p.a_pre, (const float *)p.b_pre, (float *)p.da,
-                                                      (float *)p.db, p.ebase, m.N);
+                                                      (float *)p.db, m, p.poffsets, p.ebase, p.pgate);
     else
         swiglu_bwd_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)p.a_pre,
                                                               (const __nv_bfloat16 *)p.b_pre,
-                                                              (__nv_bfloat16 *)p.da, (__nv_bfloat16 *)p.db, p.ebase,
-                                                              m.N);
+                                                              (__nv_bfloat16 *)p.da, (__nv_bfloat16 *)p.db, m,
+                                                              p.poffsets, p.ebase, p.pgate);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (launches) ++*launches;

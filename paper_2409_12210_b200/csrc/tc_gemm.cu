@@ -5,9 +5,9 @@
 // fp32 accumulator columns held in tensor memory (TMEM):
 //
 //   kind            product (per expert e, cp = padded rows, h = width)      K
-//   UpGate          Hm = silu(xp Wg^T) * (xp Wu^T)          [cp, h]          d
+//   UpGate          Hm = g * silu(xp Wg^T) * (xp Wu^T)      [cp, h]          d
 //   Down            o  = Hm Wd_e^T                          [cp, d]  fp32    h
-//   DownDgrad       dHm = dyp Wd_e -> dA, dB (SwiGLU bwd)   [cp, h]          d
+//   DownDgrad       dHm = g * (dyp Wd_e) -> dA, dB          [cp, h]          d
 //   DownWgrad       dWd_e = dyp^T Hm                        [d, h]           cp
 //   UpGateDgrad     dxp = dA Wg_e + dB Wu_e                 [cp, d]  fp32    2h
 //   UpGateWgrad     dWg_e = dA^T xp, dWu_e = dB^T xp        [h, d]           cp
@@ -21,7 +21,11 @@
 // (the instruction descriptor carries the major-ness), so the backward pass
 // needs no transposed copies.
 //
-// Activations that have the hidden axis as their width (Hm, the saved
+// (g = gate of the row's assignment: it is applied to the hidden row, in fp32,
+// before the one rounding to bf16, so neither o nor dY needs a rounded gated
+// copy; dyp is dY in group order, bit for bit.)
+//
+// Activations that have the hidden axis as their width (Hm, the saved fp32
 // pre-activations, dA, dB) are stored as panels: for expert e, panel pc holds
 // columns [64 pc, 64 pc + 64) of all cp rows contiguously, so that a single
 // two-dimensional tensor map with 128-byte rows describes the whole buffer
@@ -59,7 +63,9 @@ struct TcParams {
     const int *poffsets;
     const long long *ebase;
     int *status;
-    __nv_bfloat16 *hm, *a_pre, *b_pre, *da, *db;
+    const float *pgate;           // gate of the assignment in each padded row (0 for padding)
+    __nv_bfloat16 *hm, *da, *db;
+    float *a_pre, *b_pre;         // saved pre-activations, fp32, panel layout
     float *o, *dxp;
     __nv_bfloat16 *dw_gate, *dw_up, *dw_down;
     int save;
@@ -305,18 +311,13 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16 *dst, const float (&
     }
 }
 
-__device__ __forceinline__ void load_bf16x32(const __nv_bfloat16 *src, float (&v)[32])
+__device__ __forceinline__ void load_f32x32(const float *src, float (&v)[32])
 {
-    const uint4 *p = reinterpret_cast<const uint4 *>(src);
+    const float4 *p = reinterpret_cast<const float4 *>(src);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        const uint4 u = p[q];
-        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            v[q * 8 + 2 * i] = __uint_as_float(w[i] << 16);
-            v[q * 8 + 2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
-        }
+    for (int q = 0; q < 8; ++q) {
+        const float4 u = p[q];
+        v[4 * q] = u.x; v[4 * q + 1] = u.y; v[4 * q + 2] = u.z; v[4 * q + 3] = u.w;
     }
 }
 
@@ -334,6 +335,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
     const int d = prm.meta.d, S = prm.meta.S;
     const bool have_acc = t.nk > 0;
     if constexpr (KIND == TcUpGate) {
+        const float gate = prm.pgate[t.prow0 + t.m0 + row];
         for (int c = 0; c < t.ncols; c += 32) {
             uint32_t ra[32], rb[32];
             tmem_ld32(tacc + c, ra);
@@ -344,14 +346,14 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             for (int i = 0; i < 32; ++i) {
                 av[i] = __uint_as_float(ra[i]);
                 bv[i] = __uint_as_float(rb[i]);
-                hm[i] = av[i] * (1.0f / (1.0f + __expf(-av[i]))) * bv[i];
+                hm[i] = gate * (av[i] * (1.0f / (1.0f + __expf(-av[i]))) * bv[i]);
             }
             const int col = t.n0 + c;
             const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
             store_bf16x32(prm.hm + idx, hm);
             if (prm.save) {
-                store_bf16x32(prm.a_pre + idx, av);
-                store_bf16x32(prm.b_pre + idx, bv);
+                store_f32x32(prm.a_pre + idx, av);
+                store_f32x32(prm.b_pre + idx, bv);
             }
         }
     } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
@@ -366,6 +368,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             store_f32x32(out + c, v);
         }
     } else if constexpr (KIND == TcDownDgrad) {
+        const float gate = prm.pgate[t.prow0 + t.m0 + row];
         for (int c = 0; c < t.ncols; c += 32) {
             uint32_t r[32];
             tmem_ld32(tacc + c, r);
@@ -373,11 +376,11 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             const int col = t.n0 + c;
             const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
             float av[32], bv[32], da[32], db[32];
-            load_bf16x32(prm.a_pre + idx, av);
-            load_bf16x32(prm.b_pre + idx, bv);
+            load_f32x32(prm.a_pre + idx, av);
+            load_f32x32(prm.b_pre + idx, bv);
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const float dh = __uint_as_float(r[i]);
+                const float dh = gate * __uint_as_float(r[i]);
                 const float sg = 1.0f / (1.0f + __expf(-av[i]));
                 da[i] = dh * bv[i] * sg * (1.0f + av[i] * (1.0f - sg));
                 db[i] = dh * av[i] * sg;
@@ -653,9 +656,10 @@ TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *
     prm.poffsets = p.poffsets;
     prm.ebase = p.ebase;
     prm.status = p.status;
+    prm.pgate = p.pgate;
     prm.hm = (__nv_bfloat16 *)p.hm;
-    prm.a_pre = (__nv_bfloat16 *)p.a_pre;
-    prm.b_pre = (__nv_bfloat16 *)p.b_pre;
+    prm.a_pre = (float *)p.a_pre;
+    prm.b_pre = (float *)p.b_pre;
     prm.da = (__nv_bfloat16 *)p.da;
     prm.db = (__nv_bfloat16 *)p.db;
     prm.o = (float *)p.o;

@@ -19,9 +19,9 @@ void tc_set_force_simt(int on);
 
 // The six grouped products of the layer (Sec. 3.1, Eq. 4 and its gradient).
 enum TcKind : int {
-    TcUpGate = 0,       // Hm = silu(xp Wg^T) * (xp Wu^T), optionally saving both pre-activations
+    TcUpGate = 0,       // Hm = g * silu(xp Wg^T) * (xp Wu^T), optionally saving both pre-activations (fp32)
     TcDown = 1,         // o = Hm Wd^T into the fp32 buffer o
-    TcDownDgrad = 2,    // dHm = dyp Wd, fused SwiGLU backward -> dA, dB
+    TcDownDgrad = 2,    // dHm = g * (dyp Wd), fused SwiGLU backward -> dA, dB
     TcDownWgrad = 3,    // dWd = dyp^T Hm
     TcUpGateDgrad = 4,  // dxp = dA Wg + dB Wu into the fp32 buffer dxp
     TcUpGateWgrad = 5   // dWg = dA^T xp, dWu = dB^T xp
