@@ -19,7 +19,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -79,43 +78,71 @@ def stage_work(counts, cfg):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Reads SM clock, power and throttle reasons through NVML (read-only queries) every few
+    milliseconds while the timed region runs."""
 
     def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+        self.index, self.rows, self.stop_flag, self.thread, self.err = index, [], False, None, None
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
-            threading.Thread(target=self._read, daemon=True).start()
-        except Exception:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_sm = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:                      # no NVML: report that instead of clocks
+            self.err = f"nvml unavailable: {type(e).__name__}"
+            return
+        self.thread = threading.Thread(target=self._poll, daemon=True)
+        self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+    def _poll(self):
+        nv = self.nv
+        while not self.stop_flag:
+            try:
+                sm = float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                power = float(nv.nvmlDeviceGetPowerUsage(self.h)) / 1e3
+                self.rows.append((sm, reasons, power))
+            except Exception as e:
+                self.err = f"nvml query failed: {type(e).__name__}"
+                return
+            time.sleep(0.004)
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-                for nme, v in zip(names, r[3:7]):
-                    if v.lower().startswith("active"):
-                        reasons.add(nme)
-            except Exception:
-                pass
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        self.stop_flag = True
+        if self.thread is not None:
+            self.thread.join(timeout=1.0)
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": [self.err or "no samples"]}
+        bits = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+        seen = set()
+        for _, r, _ in self.rows:
+            for b, name in bits.items():
+                if r & b:
+                    seen.add(name)
+        return {"sm_mhz": float(np.median([r[0] for r in self.rows])), "sm_max_mhz": self.max_sm,
+                "power_w_max": max(r[2] for r in self.rows), "samples": len(self.rows), "reasons": sorted(seen)}
+
+
+def max_over_ranks(ms: float, device=None) -> float:
+    """Largest per-rank time: the job's time is the slowest replica's (no-op for one process)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Replicas process world x tokens_per_rank tokens in the time of the slowest one."""
+    return world * tokens_per_rank / (ms_per_step / 1e3)
 
 
 def cpu_oracle_sample(inp, n_tok):
@@ -165,7 +192,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="train_16k", choices=sorted(I.CONFIGS))
-    ap.add_argument("--cpu-tokens", type=int, default=48, help="tokens of the CPU baseline sample")
+    ap.add_argument("--cpu-tokens", type=int, default=64, help="tokens of the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = I.CONFIGS[args.workload]
@@ -238,12 +265,9 @@ def main():
     clocks = sampler.stop()
     ms_total = ev0.elapsed_time(ev1)
     stage_ms = layer.stage_timing_end(n_calls)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dev)
     ms_step = ms_total / K
-    value = world * T / (ms_step / 1e3)
+    value = whole_job_value(T, world, ms_step)
 
     # ---- end to end: pinned host inputs in, results out, every step ----
     hx, hdy = torch.from_numpy(inp.x).to(dt).pin_memory(), torch.from_numpy(inp.dy).to(dt).pin_memory()
@@ -269,11 +293,8 @@ def main():
     ev1.record()
     sync_all()
     ms_e2e = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * T / (ms_e2e / K / 1e3)
+    ms_e2e = max_over_ranks(ms_e2e, dev)
+    e2e_value = whole_job_value(T, world, ms_e2e / K)
 
     if rank != 0:
         if world > 1:

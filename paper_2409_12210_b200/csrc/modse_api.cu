@@ -62,8 +62,8 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
     L.hm = take(L.hb * esz);
     L.o = take((size_t)L.Pmax * m.d * 4);     // fp32 for every layer type
     if (save) {
-        L.a_pre = take(L.hb * 4);   // pre-activations are saved in fp32 by the tensor-core path
-        L.b_pre = take(L.hb * 4);
+        L.a_pre = take(L.hb * esz);   // fp32 path: pre-activations A, B; bf16 path: B*silu'(A) and silu(A)
+        L.b_pre = take(L.hb * esz);
         L.dg = take(kT * 4);
         L.dz = take(kT * 4);
         L.dwr_partial = take((size_t)L.nblk_bwd * N * m.d * 4);

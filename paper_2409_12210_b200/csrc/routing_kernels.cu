@@ -12,9 +12,9 @@
 //                      token's slots, are kept in fp32 for every layer type so
 //                      that the sum is rounded to the layer type only once.)
 //   dg_permute_kernel  dg[t,j] = <dY_t, E_(t,j)>, rows of dY in group order.
-//   router_bwd_kernel  softmax Jacobian on the kept logits, dx assembly and
-//                      per-block partial sums of dW_router; reduced in block
-//                      order by reduce_dwr_kernel so the result is reproducible.
+//   router_dx_kernel   softmax Jacobian on the kept logits and dx assembly.
+//   router_dwr_kernel  per-block partial sums of dW_router = dz^T x, reduced in
+//                      block order by reduce_dwr_kernel (reproducible).
 //
 // No kernel uses a floating-point atomic; every sum has a fixed order.
 #include "modse_internal.h"
@@ -375,88 +375,96 @@ dg_permute_kernel(const T *__restrict__ dy, const float *__restrict__ o, int Tto
 }
 
 // ---------------------------------------------------------------------------
-// Router backward.  Phase A (warp per token): s = sum_j g_j dg_j,
+// Router backward, part 1 (warp per token): s = sum_j g_j dg_j,
 // dz_j = g_j (dg_j - s), dx_t = sum_j dxp[row_j] + sum_j dz_j W_router[e_j].
-// Phase B (thread per column): partial dW_router over this block's tokens in
-// ascending token order, kept in shared memory [N][dc] and written out.
 // ---------------------------------------------------------------------------
 template <typename T, typename TO>
 __global__ void __launch_bounds__(256)
-router_bwd_kernel(const T *__restrict__ x, const T *__restrict__ w_router, const float *__restrict__ dxp,
-                  int Ttok,
-                  int d, int N, int k, int dc, const int *__restrict__ topk_idx,
-                  const float *__restrict__ topk_gate, const int *__restrict__ prow_of,
-                  const float *__restrict__ dg, float *__restrict__ dz, TO *__restrict__ dx,
-                  float *__restrict__ dwr_partial)
+router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, int Ttok, int d, int k,
+                 const int *__restrict__ topk_idx, const float *__restrict__ topk_gate,
+                 const int *__restrict__ prow_of, const float *__restrict__ dg, float *__restrict__ dz,
+                 TO *__restrict__ dx)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *dzs = reinterpret_cast<float *>(smem_raw);                    // [128][2]
-    int *idxs = reinterpret_cast<int *>(dzs + kRouterBwdTokB * 2);       // [128][2]
-    float *acc = reinterpret_cast<float *>(idxs + kRouterBwdTokB * 2);   // [N][dc]
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int t0 = blockIdx.x * kRouterBwdTokB;
-    const int c0 = blockIdx.y * dc;
-    const int cw = min(dc, d - c0);
-
-    for (int tl = warp; tl < kRouterBwdTokB; tl += 8) {
-        const int t = t0 + tl;
-        if (t >= Ttok) {
-            if (lane < 2) { dzs[tl * 2 + lane] = 0.f; idxs[tl * 2 + lane] = 0; }
-            continue;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * 8 + warp;
+    if (t >= Ttok) return;
+    float g[2] = {0.f, 0.f}, dgv[2] = {0.f, 0.f}, dzv[2];
+    int e[2] = {0, 0}, rows[2] = {-1, -1};
+    for (int j = 0; j < k; ++j) {
+        g[j] = topk_gate[(size_t)t * k + j];
+        dgv[j] = dg[(size_t)t * k + j];
+        e[j] = topk_idx[(size_t)t * k + j];
+        rows[j] = prow_of[(size_t)t * k + j];
+    }
+    const float s = g[0] * dgv[0] + g[1] * dgv[1];
+    dzv[0] = g[0] * (dgv[0] - s);
+    dzv[1] = g[1] * (dgv[1] - s);
+    if (lane < k) dz[(size_t)t * k + lane] = dzv[lane];
+    for (int c = lane * 8; c < d; c += 256) {
+        float a[8], out[8], wv[8];
+        load8(dxp + (size_t)rows[0] * d + c, out);
+        if (k > 1) {
+            load8(dxp + (size_t)rows[1] * d + c, a);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) out[u] += a[u];
         }
-        float g[2] = {0.f, 0.f}, dgv[2] = {0.f, 0.f}, dzv[2];
-        int e[2] = {0, 0}, rows[2] = {-1, -1};
         for (int j = 0; j < k; ++j) {
-            g[j] = topk_gate[(size_t)t * k + j];
-            dgv[j] = dg[(size_t)t * k + j];
-            e[j] = topk_idx[(size_t)t * k + j];
-            rows[j] = prow_of[(size_t)t * k + j];
-        }
-        const float s = g[0] * dgv[0] + g[1] * dgv[1];
-        dzv[0] = g[0] * (dgv[0] - s);
-        dzv[1] = g[1] * (dgv[1] - s);
-        if (lane < 2) {
-            dzs[tl * 2 + lane] = (lane < k) ? dzv[lane] : 0.f;
-            idxs[tl * 2 + lane] = e[lane];
-            if (blockIdx.y == 0 && lane < k) dz[(size_t)t * k + lane] = dzv[lane];
-        }
-        if (blockIdx.y == 0) {
-            for (int c = lane * 8; c < d; c += 256) {
-                float a[8], out[8], wv[8];
-                load8(dxp + (size_t)rows[0] * d + c, out);
-                if (k > 1) {
-                    load8(dxp + (size_t)rows[1] * d + c, a);
+            load8(w_router + (size_t)e[j] * d + c, wv);
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) out[u] += a[u];
-                }
-                for (int j = 0; j < k; ++j) {
-                    load8(w_router + (size_t)e[j] * d + c, wv);
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) out[u] = fmaf(dzv[j], wv[u], out[u]);
-                }
-                store8(dx + (size_t)t * d + c, out);
-            }
+            for (int u = 0; u < 8; ++u) out[u] = fmaf(dzv[j], wv[u], out[u]);
         }
+        store8(dx + (size_t)t * d + c, out);
     }
-    for (int i = tid; i < N * dc; i += 256) acc[i] = 0.f;
-    __syncthreads();
+}
+
+// ---------------------------------------------------------------------------
+// Router backward, part 2: dW_router = dz^T x as per-block partial sums.  Block
+// (bx, by) owns tokens [128 bx, +128) and columns [256 by, +256); each thread
+// owns one column and adds its tokens in ascending order, eight experts at a
+// time, against the dense [128][8] slice of dz held in shared memory.
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int *__restrict__ topk_idx,
+                  const float *__restrict__ dz, float *__restrict__ dwr_partial)
+{
+    __shared__ float dzs[kRouterBwdTokB][8];
+    __shared__ int idxs[kRouterBwdTokB][2];
+    __shared__ float dzk[kRouterBwdTokB][2];
+    const int tid = threadIdx.x;
+    const int t0 = blockIdx.x * kRouterBwdTokB;
+    const int c = blockIdx.y * 256 + tid;
     const int ntok = min(kRouterBwdTokB, Ttok - t0);
-    for (int c = tid; c < cw; c += 256) {
-        for (int tl = 0; tl < ntok; ++tl) {
-            float xv;
-            if (sizeof(T) == 4) xv = reinterpret_cast<const float *>(x)[(size_t)(t0 + tl) * d + c0 + c];
-            else xv = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(x)[(size_t)(t0 + tl) * d + c0 + c]);
-            for (int j = 0; j < k; ++j) {
-                float *a = &acc[idxs[tl * 2 + j] * dc + c];
-                *a = fmaf(dzs[tl * 2 + j], xv, *a);
-            }
-        }
+    for (int i = tid; i < kRouterBwdTokB * 2; i += 256) {
+        const int tl = i >> 1, j = i & 1;
+        const bool ok = tl < ntok && j < k;
+        idxs[tl][j] = ok ? topk_idx[(size_t)(t0 + tl) * k + j] : -1;
+        dzk[tl][j] = ok ? dz[(size_t)(t0 + tl) * k + j] : 0.f;
     }
-    __syncthreads();
-    for (int i = tid; i < N * cw; i += 256) {
-        const int e = i / cw, c = i % cw;
-        dwr_partial[((size_t)blockIdx.x * N + e) * d + c0 + c] = acc[e * dc + c];
+    for (int g0 = 0; g0 < N; g0 += 8) {
+        __syncthreads();
+        for (int i = tid; i < kRouterBwdTokB * 8; i += 256) {
+            const int tl = i >> 3, e = g0 + (i & 7);
+            float v = 0.f;
+            if (idxs[tl][0] == e) v = dzk[tl][0];
+            if (idxs[tl][1] == e) v = dzk[tl][1];
+            dzs[tl][i & 7] = v;
+        }
+        __syncthreads();
+        if (c < d) {
+            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+            for (int tl = 0; tl < ntok; ++tl) {
+                float xv;
+                if (sizeof(T) == 4) xv = reinterpret_cast<const float *>(x)[(size_t)(t0 + tl) * d + c];
+                else xv = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(x)[(size_t)(t0 + tl) * d + c]);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) acc[i] = fmaf(dzs[tl][i], xv, acc[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (g0 + i < N) dwr_partial[((size_t)blockIdx.x * N + g0 + i) * d + c] = acc[i];
+        }
     }
 }
 
@@ -566,34 +574,31 @@ cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *
     return cudaSuccess;
 }
 
-template <typename T, typename TO>
-static cudaError_t run_router_bwd(dim3 grid, size_t smem, cudaStream_t s, const LayerMeta &m, const void *x,
-                                  const void *w_router, int T_tok, int dc, const WsPtrs &p, void *dx)
-{
-    auto kern = router_bwd_kernel<T, TO>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, 256, smem, s>>>((const T *)x, (const T *)w_router, (const float *)p.dxp, T_tok, m.d, m.N, m.k, dc,
-                                 p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz, (TO *)dx, p.dwr_partial);
-    return cudaSuccess;
-}
-
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
                               int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
                               cudaStream_t s, int *launches)
 {
-    // column chunk so that the [N][dc] fp32 accumulator fits in 64 KB of shared memory
-    int dc = m.d;
-    while ((size_t)m.N * dc * 4 > 64 * 1024 && dc > 8) dc = (dc / 2 + 7) & ~7;
-    const int ychunks = (m.d + dc - 1) / dc;
-    const size_t smem =
-        sizeof(float) * kRouterBwdTokB * 2 + sizeof(int) * kRouterBwdTokB * 2 + sizeof(float) * m.N * dc;
-    dim3 grid(nblk_bwd, ychunks);
-    cudaError_t re;
-    if (dt == MODSE_F32) re = run_router_bwd<float, float>(grid, smem, s, m, x, w_router, T, dc, p, dx);
-    else if (out_f32) re = run_router_bwd<__nv_bfloat16, float>(grid, smem, s, m, x, w_router, T, dc, p, dx);
-    else re = run_router_bwd<__nv_bfloat16, __nv_bfloat16>(grid, smem, s, m, x, w_router, T, dc, p, dx);
-    if (re != cudaSuccess) return re;
+    const int grid_dx = (T + 7) / 8;
+    const float *dxp = (const float *)p.dxp;
+    if (dt == MODSE_F32)
+        router_dx_kernel<float, float><<<grid_dx, 256, 0, s>>>((const float *)w_router, dxp, T, m.d, m.k, p.topk_idx,
+                                                               p.topk_gate, p.prow_of, p.dg, p.dz, (float *)dx);
+    else if (out_f32)
+        router_dx_kernel<__nv_bfloat16, float><<<grid_dx, 256, 0, s>>>((const __nv_bfloat16 *)w_router, dxp, T, m.d,
+                                                                       m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg,
+                                                                       p.dz, (float *)dx);
+    else
+        router_dx_kernel<__nv_bfloat16, __nv_bfloat16><<<grid_dx, 256, 0, s>>>(
+            (const __nv_bfloat16 *)w_router, dxp, T, m.d, m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz,
+            (__nv_bfloat16 *)dx);
+    MODSE_LAUNCH_CHECK();
+    dim3 grid(nblk_bwd, (m.d + 255) / 256);
+    if (dt == MODSE_F32)
+        router_dwr_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.topk_idx, p.dz,
+                                                      p.dwr_partial);
+    else
+        router_dwr_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k, p.topk_idx,
+                                                              p.dz, p.dwr_partial);
     MODSE_LAUNCH_CHECK();
     const int n = m.N * m.d;
     reduce_dwr_kernel<<<(n + 255) / 256, 256, 0, s>>>(p.dwr_partial, nblk_bwd, n, dw_router);

@@ -12,11 +12,12 @@
 //   UpGateDgrad     dxp = dA Wg_e + dB Wu_e                 [cp, d]  fp32    2h
 //   UpGateWgrad     dWg_e = dA^T xp, dWu_e = dB^T xp        [h, d]           cp
 //
-// Roles inside a CTA (192 threads): warp 0 issues TMA loads into a 4-stage
+// Roles inside a CTA (320 threads): warp 0 issues TMA loads into a 4-stage
 // shared-memory ring (every box is 64 elements x 64 rows, 128-byte swizzle),
 // warp 1 issues tcgen05.mma with the accumulator in TMEM (two accumulators, so
-// the epilogue of one tile overlaps the main loop of the next), warps 2-5 read
-// the accumulator with tcgen05.ld and run the fused epilogue.  Operands are
+// the epilogue of one tile overlaps the main loop of the next), warps 2-9 read
+// the accumulator with tcgen05.ld (two warps per TMEM lane quadrant, each half
+// of the columns) and run the fused epilogue.  Operands are
 // consumed either K-major or MN-major straight from their row-major buffers
 // (the instruction descriptor carries the major-ness), so the backward pass
 // needs no transposed copies.
@@ -25,8 +26,12 @@
 // before the one rounding to bf16, so neither o nor dY needs a rounded gated
 // copy; dyp is dY in group order, bit for bit.)
 //
-// Activations that have the hidden axis as their width (Hm, the saved fp32
-// pre-activations, dA, dB) are stored as panels: for expert e, panel pc holds
+// For backward the up/gate epilogue saves, from its fp32 accumulators A and B,
+// sp = B * silu'(A) and sq = silu(A) (bf16): then dA = dHm * sp, dB = dHm * sq, one
+// rounded factor each instead of two rounded pre-activations.
+//
+// Activations that have the hidden axis as their width (Hm, sp, sq, dA, dB)
+// are stored as panels: for expert e, panel pc holds
 // columns [64 pc, 64 pc + 64) of all cp rows contiguously, so that a single
 // two-dimensional tensor map with 128-byte rows describes the whole buffer
 // although the row length h differs from expert to expert.
@@ -53,7 +58,7 @@ constexpr int kBoxBytes = 64 * 64 * 2;           // one TMA box: 64 rows of 128 
 constexpr int kARegion = 2 * kBoxBytes;          // 128 rows (or 128 MN elements) x 64 K
 constexpr int kBRegion = 4 * kBoxBytes;          // up to 256 rows x 64 K
 constexpr int kStageBytes = kARegion + kBRegion; // 48 KB
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;                   // TMA warp, MMA warp, eight epilogue warps
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
@@ -65,7 +70,7 @@ struct TcParams {
     int *status;
     const float *pgate;           // gate of the assignment in each padded row (0 for padding)
     __nv_bfloat16 *hm, *da, *db;
-    float *a_pre, *b_pre;         // saved pre-activations, fp32, panel layout
+    __nv_bfloat16 *sp, *sq;       // saved for backward: sp = B * silu'(A), sq = silu(A) (panel layout)
     float *o, *dxp;
     __nv_bfloat16 *dw_gate, *dw_up, *dw_down;
     int save;
@@ -311,16 +316,6 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16 *dst, const float (&
     }
 }
 
-__device__ __forceinline__ void load_f32x32(const float *src, float (&v)[32])
-{
-    const float4 *p = reinterpret_cast<const float4 *>(src);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-        const float4 u = p[q];
-        v[4 * q] = u.x; v[4 * q + 1] = u.y; v[4 * q + 2] = u.z; v[4 * q + 3] = u.w;
-    }
-}
-
 __device__ __forceinline__ void store_f32x32(float *dst, const float (&v)[32])
 {
     float4 *p = reinterpret_cast<float4 *>(dst);
@@ -328,37 +323,50 @@ __device__ __forceinline__ void store_f32x32(float *dst, const float (&v)[32])
     for (int q = 0; q < 8; ++q) p[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
 }
 
-// Epilogue of one tile for one thread (= one accumulator row).
+// Epilogue of one tile for one thread: accumulator row `row`, columns [c_begin, c_end).
 template <int KIND>
-__device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t, uint32_t tacc, int row)
+__device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t, uint32_t tacc, int row, int c_begin,
+                                             int c_end)
 {
     const int d = prm.meta.d, S = prm.meta.S;
     const bool have_acc = t.nk > 0;
+    auto panel_index = [&](int c) {
+        const int col = t.n0 + c;
+        return ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
+    };
     if constexpr (KIND == TcUpGate) {
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
-        for (int c = 0; c < t.ncols; c += 32) {
+        for (int c = c_begin; c < c_end; c += 32) {
             uint32_t ra[32], rb[32];
             tmem_ld32(tacc + c, ra);
             tmem_ld32(tacc + t.ncols + c, rb);
             tmem_ld_wait();
-            float hm[32], av[32], bv[32];
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                av[i] = __uint_as_float(ra[i]);
-                bv[i] = __uint_as_float(rb[i]);
-                hm[i] = gate * (av[i] * (1.0f / (1.0f + __expf(-av[i]))) * bv[i]);
-            }
-            const int col = t.n0 + c;
-            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
-            store_bf16x32(prm.hm + idx, hm);
+            const size_t idx = panel_index(c);
+            float hm[32];
             if (prm.save) {
-                store_f32x32(prm.a_pre + idx, av);
-                store_f32x32(prm.b_pre + idx, bv);
+                float sp[32], sq[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float av = __uint_as_float(ra[i]), bv = __uint_as_float(rb[i]);
+                    const float sg = 1.0f / (1.0f + __expf(-av));
+                    sq[i] = av * sg;
+                    sp[i] = bv * sg * (1.0f + av * (1.0f - sg));
+                    hm[i] = gate * (sq[i] * bv);
+                }
+                store_bf16x32(prm.sp + idx, sp);
+                store_bf16x32(prm.sq + idx, sq);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const float av = __uint_as_float(ra[i]), bv = __uint_as_float(rb[i]);
+                    hm[i] = gate * (av * (1.0f / (1.0f + __expf(-av))) * bv);
+                }
             }
+            store_bf16x32(prm.hm + idx, hm);
         }
     } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
         float *out = (KIND == TcDown ? prm.o : prm.dxp) + (size_t)(t.prow0 + t.m0 + row) * d + t.n0;
-        for (int c = 0; c < t.ncols; c += 32) {
+        for (int c = c_begin; c < c_end; c += 32) {
             uint32_t r[32];
             float v[32];
             tmem_ld32(tacc + c, r);
@@ -368,29 +376,56 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             store_f32x32(out + c, v);
         }
     } else if constexpr (KIND == TcDownDgrad) {
+        // dA = dHm * sp, dB = dHm * sq with dHm = gate * acc; the saved factors of the next
+        // chunk are fetched while this one is computed
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
-        for (int c = 0; c < t.ncols; c += 32) {
+        uint4 praw[4], qraw[4];
+        {
+            const size_t idx = panel_index(c_begin);
+            const uint4 *pp = reinterpret_cast<const uint4 *>(prm.sp + idx);
+            const uint4 *qq = reinterpret_cast<const uint4 *>(prm.sq + idx);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { praw[i] = pp[i]; qraw[i] = qq[i]; }
+        }
+        for (int c = c_begin; c < c_end; c += 32) {
             uint32_t r[32];
             tmem_ld32(tacc + c, r);
-            tmem_ld_wait();
-            const int col = t.n0 + c;
-            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
-            float av[32], bv[32], da[32], db[32];
-            load_f32x32(prm.a_pre + idx, av);
-            load_f32x32(prm.b_pre + idx, bv);
+            uint4 pn[4], qn[4];
+            const bool more = c + 32 < c_end;
+            if (more) {
+                const size_t nidx = panel_index(c + 32);
+                const uint4 *pp = reinterpret_cast<const uint4 *>(prm.sp + nidx);
+                const uint4 *qq = reinterpret_cast<const uint4 *>(prm.sq + nidx);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float dh = gate * __uint_as_float(r[i]);
-                const float sg = 1.0f / (1.0f + __expf(-av[i]));
-                da[i] = dh * bv[i] * sg * (1.0f + av[i] * (1.0f - sg));
-                db[i] = dh * av[i] * sg;
+                for (int i = 0; i < 4; ++i) { pn[i] = pp[i]; qn[i] = qq[i]; }
+            }
+            tmem_ld_wait();
+            const size_t idx = panel_index(c);
+            float da[32], db[32];
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+                const uint32_t pw[4] = {praw[q4].x, praw[q4].y, praw[q4].z, praw[q4].w};
+                const uint32_t qw[4] = {qraw[q4].x, qraw[q4].y, qraw[q4].z, qraw[q4].w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int e0 = q4 * 8 + 2 * i;
+                    const float dh0 = gate * __uint_as_float(r[e0]), dh1 = gate * __uint_as_float(r[e0 + 1]);
+                    da[e0] = dh0 * __uint_as_float(pw[i] << 16);
+                    da[e0 + 1] = dh1 * __uint_as_float(pw[i] & 0xFFFF0000u);
+                    db[e0] = dh0 * __uint_as_float(qw[i] << 16);
+                    db[e0 + 1] = dh1 * __uint_as_float(qw[i] & 0xFFFF0000u);
+                }
             }
             store_bf16x32(prm.da + idx, da);
             store_bf16x32(prm.db + idx, db);
+            if (more) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) { praw[i] = pn[i]; qraw[i] = qn[i]; }
+            }
         }
     } else if constexpr (KIND == TcDownWgrad) {
         const size_t oidx = (size_t)(t.m0 + row) * S + t.ho + t.n0;
-        for (int c = 0; c < t.ncols; c += 32) {
+        for (int c = c_begin; c < c_end; c += 32) {
             float v[32];
             if (have_acc) {
                 uint32_t r[32];
@@ -408,7 +443,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
     } else {
         __nv_bfloat16 *obase = t.which ? prm.dw_up : prm.dw_gate;
         const size_t oidx = (size_t)(t.ho + t.m0 + row) * d + t.n0;
-        for (int c = 0; c < t.ncols; c += 32) {
+        for (int c = c_begin; c < c_end; c += 32) {
             float v[32];
             if (have_acc) {
                 uint32_t r[32];
@@ -458,7 +493,7 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(smem_u32(&st->tmem_full[a]), 1);
-            mbar_init(smem_u32(&st->tmem_empty[a]), 128);
+            mbar_init(smem_u32(&st->tmem_empty[a]), 256);
         }
         st->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -561,8 +596,9 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
             }
         }
     } else {
-        // ===================== epilogue (warps 2..5) =====================
+        // ===================== epilogue (warps 2..9) =====================
         const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
+        const int half = (warp - 2) >> 2;          // which half of the tile's columns
         const int row = quad * 32 + lane;
         int cursor = 0, it = 0;
         bool ok = true;
@@ -573,7 +609,8 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
             if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, prm.status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
-            epilogue_row<KIND>(prm, t, tacc, row);
+            const int chalf = t.ncols >> 1;            // a multiple of 32: ncols is a multiple of 64
+            epilogue_row<KIND>(prm, t, tacc, row, half * chalf, (half + 1) * chalf);
             tc_fence_before();
             mbar_arrive(smem_u32(&st->tmem_empty[acc]));
         }
@@ -658,8 +695,8 @@ TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *
     prm.status = p.status;
     prm.pgate = p.pgate;
     prm.hm = (__nv_bfloat16 *)p.hm;
-    prm.a_pre = (float *)p.a_pre;
-    prm.b_pre = (float *)p.b_pre;
+    prm.sp = (__nv_bfloat16 *)p.a_pre;
+    prm.sq = (__nv_bfloat16 *)p.b_pre;
     prm.da = (__nv_bfloat16 *)p.da;
     prm.db = (__nv_bfloat16 *)p.db;
     prm.o = (float *)p.o;

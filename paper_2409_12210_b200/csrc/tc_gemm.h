@@ -19,7 +19,7 @@ void tc_set_force_simt(int on);
 
 // The six grouped products of the layer (Sec. 3.1, Eq. 4 and its gradient).
 enum TcKind : int {
-    TcUpGate = 0,       // Hm = g * silu(xp Wg^T) * (xp Wu^T), optionally saving both pre-activations (fp32)
+    TcUpGate = 0,       // Hm = g * silu(xp Wg^T) * (xp Wu^T), optionally saving B*silu'(A) and silu(A)
     TcDown = 1,         // o = Hm Wd^T into the fp32 buffer o
     TcDownDgrad = 2,    // dHm = g * (dyp Wd), fused SwiGLU backward -> dA, dB
     TcDownWgrad = 3,    // dWd = dyp^T Hm
