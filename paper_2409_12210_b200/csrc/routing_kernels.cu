@@ -170,6 +170,117 @@ router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok,
 }
 
 // ---------------------------------------------------------------------------
+// Router, bf16 with at most 16 experts: the logits of 16 tokens per warp come
+// from mma.sync m16n8k16 (bf16 x bf16 -> fp32) fed straight from global memory.
+// A lane loads 8 consecutive elements (16 bytes) of two token rows and of one
+// router row per k-chunk of 32 and uses them as the operands of two MMAs: the
+// sum over k does not depend on which k index sits in which operand slot as
+// long as A and B agree, so no data is rearranged.  Four lanes then hold the
+// logits of one token; top-k and the gates are computed with quad shuffles.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ void quad_argmax(float &bv, int &bi)
+{
+#pragma unroll
+    for (int o = 1; o <= 2; o <<= 1) {
+        const float ov = __shfl_xor_sync(0xFFFFFFFFu, bv, o);
+        const int oi = __shfl_xor_sync(0xFFFFFFFFu, bi, o);
+        if (oi != kNoIndex && (bi == kNoIndex || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
+    }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(128)
+router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w_router, int Ttok, int d,
+                  int N, int k, int *__restrict__ topk_idx, float *__restrict__ topk_gate,
+                  int *__restrict__ block_counts)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    int *cnt = reinterpret_cast<int *>(smem_raw);                                   // [k*N], padded to 128 bytes
+    __nv_bfloat16 *wsm = reinterpret_cast<__nv_bfloat16 *>(smem_raw + 128);         // [NT*8][d + 8]
+    const int ldw = d + 8;                                                          // 16-byte skew: conflict-free rows
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, tq = lane & 3;
+    for (int i = tid; i < k * N; i += 128) cnt[i] = 0;
+    for (int i = tid * 8; i < NT * 8 * d; i += 128 * 8) {
+        const int r = i / d, c = i % d;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (r < N) v = *reinterpret_cast<const uint4 *>(w_router + (size_t)r * d + c);
+        *reinterpret_cast<uint4 *>(wsm + (size_t)r * ldw + c) = v;
+    }
+    __syncthreads();
+
+    const int t0 = blockIdx.x * kRouterTokB + warp * 16;
+    const int r0 = t0 + g, r1 = t0 + g + 8;
+    const bool v0 = r0 < Ttok, v1 = r1 < Ttok;
+    const uint4 *x0 = reinterpret_cast<const uint4 *>(x + (size_t)(v0 ? r0 : 0) * d + tq * 8);
+    const uint4 *x1 = reinterpret_cast<const uint4 *>(x + (size_t)(v1 ? r1 : 0) * d + tq * 8);
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+#pragma unroll 4
+    for (int c0 = 0; c0 < d; c0 += 32) {
+        const uint4 za = make_uint4(0u, 0u, 0u, 0u);
+        const uint4 xa = v0 ? x0[c0 >> 3] : za;     // 32 elements = 4 uint4 per row chunk; this lane's is index c0/8 + (tq folded into base)
+        const uint4 xb = v1 ? x1[c0 >> 3] : za;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const uint4 w = *reinterpret_cast<const uint4 *>(wsm + (size_t)(nt * 8 + g) * ldw + c0 + tq * 8);
+            mma_bf16_16816(acc[nt], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
+            mma_bf16_16816(acc[nt], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+        }
+    }
+    // acc[nt][0..1]: token r0, experts nt*8 + 2tq, +1;  acc[nt][2..3]: token r1, same experts
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        const int t = half ? r1 : r0;
+        float zsel[2] = {0.f, 0.f};
+        int isel[2] = {kNoIndex, kNoIndex};
+        for (int j = 0; j < k; ++j) {
+            float bv = -INFINITY;
+            int bi = kNoIndex;
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int e = nt * 8 + 2 * tq + u;
+                    const float v = acc[nt][2 * half + u];
+                    const bool usable = e < N && !(j > 0 && e == isel[0]);
+                    if (usable && (bi == kNoIndex || v > bv)) { bv = v; bi = e; }
+                }
+            quad_argmax(bv, bi);
+            zsel[j] = bv;
+            isel[j] = bi;
+        }
+        if (tq == 0 && t < Ttok) {
+            if (k == 1) {
+                topk_idx[t] = isel[0];
+                topk_gate[t] = 1.0f;
+                atomicAdd(&cnt[isel[0]], 1);
+            } else {
+                const float w1 = expf(zsel[1] - zsel[0]);
+                const float den = 1.0f + w1;
+                topk_idx[2 * (size_t)t] = isel[0];
+                topk_idx[2 * (size_t)t + 1] = isel[1];
+                topk_gate[2 * (size_t)t] = 1.0f / den;
+                topk_gate[2 * (size_t)t + 1] = w1 / den;
+                atomicAdd(&cnt[isel[0]], 1);
+                atomicAdd(&cnt[N + isel[1]], 1);
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < k * N; i += 128) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
+}
+
+// ---------------------------------------------------------------------------
 // Rank: block b owns tokens [b*64, b*64+64).  It sums the histograms of the
 // blocks before it (tokens before its own), scans the totals over experts, and
 // ranks its own assignments by token index.  Integer work only.
@@ -494,6 +605,19 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
                           const WsPtrs &p, cudaStream_t s, int *launches)
 {
     const int nblk = (T + kRouterTokB - 1) / kRouterTokB;
+    if (dt == MODSE_BF16 && m.N <= 16 && m.d % 32 == 0 && m.k * m.N * 4 <= 128) {
+        const int nt = (m.N + 7) / 8;
+        const size_t smem = 128 + (size_t)nt * 8 * (m.d + 8) * 2;
+        if (smem <= 200 * 1024) {
+            auto kern = nt == 1 ? router_mma_kernel<1> : router_mma_kernel<2>;
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            kern<<<nblk, 128, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
+                                         p.topk_idx, p.topk_gate, p.block_counts);
+            MODSE_LAUNCH_CHECK();
+            return cudaSuccess;
+        }
+    }
     const size_t esz = dt == MODSE_F32 ? 4 : 2;
     const size_t base = sizeof(int) * ((m.k * m.N + 3) & ~3) + sizeof(float) * 8 * ((m.N + 3) & ~3);
     const size_t wbytes = (size_t)m.N * m.d * esz;

@@ -238,7 +238,13 @@ __device__ __forceinline__ Tile decode_tile(const TcParams &prm, const SmemTail 
     int mt, nt, nk;
     expert_shape<KIND>(t.cp, t.h, d, mt, nt, nk);
     const int local = tile - st->tstart[cursor];
-    const int mb = local % mt, nb = local / mt;
+    // Order of an expert's tiles (the ~148 tiles in flight should share operands through L2):
+    // row-block fastest where the column operand is the big one (weights of the up/gate GEMM, Hm
+    // panels of the down wgrad), column-block fastest where all column blocks of one row block
+    // fit in flight at once (d / 256 = 8 column blocks), so the row operand is read once.
+    constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
+    const int mb = n_fastest ? local / nt : local % mt;
+    const int nb = n_fastest ? local % nt : local / mt;
     t.nk = nk;
     t.which = 0;
     t.mrows = 128;
