@@ -194,6 +194,8 @@ def main():
     ap.add_argument("--workload", default="train_16k", choices=sorted(I.CONFIGS))
     ap.add_argument("--cpu-tokens", type=int, default=64, help="tokens of the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--pair-mask", type=int, default=None,
+                    help="tuning: which grouped products use the two-SM kernel (bit per product)")
     args = ap.parse_args()
     cfg = I.CONFIGS[args.workload]
     if args.impl == "reference":
@@ -213,6 +215,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     lib_build.build()
+    if args.pair_mask is not None:
+        B.debug_set_pair_kernels(args.pair_mask)
     dev = torch.device("cuda", local_rank)
 
     inp = I.generate(cfg)

@@ -178,6 +178,13 @@ const char *modse_stage_name(int stage);
  * be called with save_for_backward = 1.  Off by default.                    */
 void modse_debug_use_fma_path(int on);
 
+/* Tuning aid, process-wide: bit k of `mask` selects, for grouped product k
+ * (0 up/gate, 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate dgrad, 5 up/gate
+ * wgrad), the kernel that computes 256-row tiles on pairs of SMs instead of
+ * 128-row tiles on single SMs.  Results are the same up to fp32 summation
+ * order inside the tensor cores.                                            */
+void modse_debug_set_pair_kernels(int mask);
+
 #ifdef __cplusplus
 }
 #endif

@@ -92,6 +92,8 @@ def load():
     lib.modse_stage_timing_end.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ip]
     lib.modse_stage_name.restype = ctypes.c_char_p
     lib.modse_stage_name.argtypes = [ci]
+    lib.modse_debug_set_pair_kernels.restype = None
+    lib.modse_debug_set_pair_kernels.argtypes = [ci]
     lib.modse_debug_use_fma_path.restype = None
     lib.modse_debug_use_fma_path.argtypes = [ci]
     _lib = lib
@@ -104,6 +106,10 @@ def status_string(status: int) -> str:
 
 def stage_name(i: int) -> str:
     return load().modse_stage_name(int(i)).decode()
+
+
+def debug_set_pair_kernels(mask: int) -> None:
+    load().modse_debug_set_pair_kernels(int(mask))
 
 
 def debug_use_fma_path(on: bool) -> None:

@@ -437,6 +437,8 @@ modse_status_t modse_set_output_f32(modse_layer_t *layer, int on)
 
 void modse_debug_use_fma_path(int on) { tc_set_force_simt(on); }
 
+void modse_debug_set_pair_kernels(int mask) { tc_set_pair_mask(mask); }
+
 const char *modse_stage_name(int stage)
 {
     static const char *names[MODSE_N_STAGES] = {"router", "rank", "permute", "upgate_gemm_swiglu", "down_gemm",

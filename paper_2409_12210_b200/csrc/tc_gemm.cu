@@ -48,6 +48,10 @@
 namespace modse {
 
 static int g_force_simt = 0;
+static int g_pair_mask = 0;      // bit k: product kind k runs on the two-CTA kernel
+void tc_set_pair_mask(int mask) { g_pair_mask = mask & 63; }
+int tc_pair_mask() { return g_pair_mask; }
+
 bool tc_force_simt() { return g_force_simt != 0; }
 void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
 
@@ -209,6 +213,7 @@ struct Tile {
     int e, cp, h, ho, prow0, pbase;   // expert, padded rows, width, width offset, first padded row, first panel row
     int m0, n0, mrows, ncols, nk, which;
     int n_mma, a_boxes, b_boxes;
+    int a_boxes_peer, b_off;          // two-CTA tiles only: boxes of the partner's rows, this CTA's column offset
 };
 
 // tiles (rows, columns) and K blocks of one expert
@@ -632,6 +637,360 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
     }
 }
 
+// ===========================================================================
+// Two-CTA variant (cta_group::2).  A cluster of two CTAs on neighbouring SMs
+// computes one 256-row tile: each CTA stages its own 128 rows of the row
+// operand and HALF of the column operand (so a CTA moves 32 KB per k-block
+// instead of 48 KB), the leader CTA (cluster rank 0) issues tcgen05.mma with
+// M = 256 reading both CTAs' shared memory, and each CTA's TMEM receives the
+// accumulator rows of its own half.  Barrier protocol:
+//   full[s]       leader only; its producer posts the byte count of both CTAs,
+//                 both producers' TMA loads complete on it
+//   empty[s]      one per CTA; tcgen05.commit multicasts to both
+//   tmem_full[a]  one per CTA; tcgen05.commit multicasts to both
+//   tmem_empty[a] leader only; one arrival per epilogue warp of both CTAs
+// ===========================================================================
+constexpr int kStages2 = 6;
+constexpr int kARegion2 = 2 * kBoxBytes;
+constexpr int kBRegion2 = 2 * kBoxBytes;
+constexpr int kStageBytes2 = kARegion2 + kBRegion2;   // 32 KB
+struct SmemTail2 {
+    unsigned long long full[kStages2], empty[kStages2], tmem_full[2], tmem_empty[2];
+    unsigned int tmem_base;
+    int abort_flag;
+    int order[kMaxExperts];
+    int key[kMaxExperts];
+    int ntile[kMaxExperts];
+    int tstart[kMaxExperts + 1];
+};
+constexpr size_t kSmemBytes2 = 1024 + (size_t)kStages2 * kStageBytes2 + sizeof(SmemTail2);
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(leader_bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ uint32_t make_idesc_pair(bool a_mn, bool b_mn, int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+}
+
+template <int KIND>
+__device__ __forceinline__ void expert_shape2(int cp, int h, int d, int &mt, int &nt, int &nk)
+{
+    if constexpr (KIND == TcUpGate)      { mt = (cp + 255) / 256; nt = (h + 127) / 128; nk = d / 64; }
+    if constexpr (KIND == TcDown)        { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = h / 64; }
+    if constexpr (KIND == TcDownDgrad)   { mt = (cp + 255) / 256; nt = (h + 255) / 256; nk = d / 64; }
+    if constexpr (KIND == TcDownWgrad)   { mt = (d + 255) / 256;  nt = (h + 255) / 256; nk = cp / 64; }
+    if constexpr (KIND == TcUpGateDgrad) { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = 2 * (h / 64); }
+    if constexpr (KIND == TcUpGateWgrad) { mt = 2 * ((h + 255) / 256); nt = (d + 255) / 256; nk = cp / 64; }
+}
+
+// Tile of this CTA (cluster rank `rank`) inside pair tile `tile`.  Fields as in the one-CTA
+// decode; m0 / mrows / a_boxes describe this CTA's 128-row half, a_boxes_peer the other half,
+// b_boxes and b_off this CTA's half of the column operand, ncols the columns that are stored.
+template <int KIND>
+__device__ __forceinline__ Tile decode_tile2(const TcParams &prm, const SmemTail2 *st, int tile, int &cursor, int rank)
+{
+    const int N = prm.meta.N, d = prm.meta.d;
+    while (cursor + 1 < N && tile >= st->tstart[cursor + 1]) ++cursor;
+    Tile t;
+    t.e = st->order[cursor];
+    t.ho = prm.meta.hoff[t.e];
+    t.h = prm.meta.hoff[t.e + 1] - t.ho;
+    t.prow0 = prm.poffsets[t.e];
+    t.cp = prm.poffsets[t.e + 1] - t.prow0;
+    t.pbase = (int)(prm.ebase[t.e] >> 6);
+    int mt, nt, nk;
+    expert_shape2<KIND>(t.cp, t.h, d, mt, nt, nk);
+    const int local = tile - st->tstart[cursor];
+    constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
+    int mb = n_fastest ? local / nt : local % mt;
+    const int nb = n_fastest ? local % nt : local / mt;
+    t.nk = nk;
+    t.which = 0;
+    int row_extent;                       // extent of the tile's row dimension for this expert
+    if constexpr (KIND == TcDownWgrad) row_extent = d;
+    else if constexpr (KIND == TcUpGateWgrad) { row_extent = t.h; t.which = mb & 1; mb >>= 1; }
+    else row_extent = t.cp;
+    const int m_pair = mb * 256;
+    t.m0 = m_pair + 128 * rank;
+    t.mrows = max(0, min(128, row_extent - t.m0));
+    const int peer_rows = max(0, min(128, row_extent - (m_pair + 128 * (1 - rank))));
+    t.a_boxes = t.mrows / 64;
+    t.a_boxes_peer = peer_rows / 64;
+    if constexpr (KIND == TcUpGate) {
+        t.n0 = nb * 128; t.ncols = min(128, t.h - t.n0);
+        t.n_mma = 2 * t.ncols; t.b_boxes = t.ncols / 64; t.b_off = 0;
+    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad) {
+        t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
+        t.n_mma = t.ncols; t.b_boxes = t.ncols / 128; t.b_off = rank * (t.ncols / 2);
+    } else {
+        t.n0 = nb * 256; t.ncols = min(256, t.h - t.n0);
+        t.n_mma = (t.ncols + 127) & ~127; t.b_boxes = t.n_mma / 128; t.b_off = rank * (t.n_mma / 2);
+    }
+    return t;
+}
+
+template <int KIND>
+__device__ __forceinline__ void issue_loads2(const TcMaps &maps, const Tile &t, int rank, int kb, uint32_t a_dst,
+                                             uint32_t b_dst, uint32_t bar)
+{
+    if constexpr (KIND == TcUpGate) {
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.xp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        const CUtensorMap *bm = rank ? &maps.wup : &maps.wgate;     // gate columns live in CTA 0, up columns in CTA 1
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d_pair(b_dst + i * kBoxBytes, bm, bar, kb * 64, t.ho + t.n0 + 64 * i);
+    } else if constexpr (KIND == TcDown) {
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + kb * t.cp + t.m0 + 64 * i);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + kb * 64, t.n0 + t.b_off + 64 * i);
+    } else if constexpr (KIND == TcDownDgrad) {
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.dyp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + t.b_off + 64 * i, kb * 64);
+    } else if constexpr (KIND == TcDownWgrad) {
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.hm, bar, 0,
+                             t.pbase + ((t.n0 + t.b_off) / 64 + i) * t.cp + kb * 64);
+    } else if constexpr (KIND == TcUpGateDgrad) {
+        const int half = t.h / 64;
+        const bool second = kb >= half;
+        const int kk = second ? kb - half : kb;
+        const CUtensorMap *am = second ? &maps.db : &maps.da;
+        const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d_pair(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + kk * t.cp + t.m0 + 64 * i);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d_pair(b_dst + i * kBoxBytes, bm, bar, t.n0 + t.b_off + 64 * i, t.ho + kk * 64);
+    } else {
+        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d_pair(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.xp, bar, t.n0 + t.b_off + 64 * i, t.prow0 + kb * 64);
+    }
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_grouped_gemm_pair(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
+    unsigned char *smem = smem_raw + pad;
+    const uint32_t stage_base = raw + pad;
+    SmemTail2 *st = reinterpret_cast<SmemTail2 *>(smem + (size_t)kStages2 * kStageBytes2);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int N = prm.meta.N, d = prm.meta.d;
+    const int rank = (int)cluster_ctarank();
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+    for (int e = tid; e < N; e += kThreads) {
+        const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
+        const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
+        int mt, nt, nk;
+        expert_shape2<KIND>(cp, h, d, mt, nt, nk);
+        st->ntile[e] = mt * nt;
+        st->key[e] = nk;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kStages2; ++s) {
+            mbar_init(smem_u32(&st->full[s]), 1);
+            mbar_init(smem_u32(&st->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&st->tmem_full[a]), 1);
+            mbar_init(smem_u32(&st->tmem_empty[a]), 16);      // 8 epilogue warps of each of the two CTAs
+        }
+        st->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    for (int e = tid; e < N; e += kThreads) {
+        int rk = 0;
+        const int ke = st->key[e];
+        for (int f = 0; f < N; ++f) {
+            const int kf = st->key[f];
+            rk += (kf > ke) || (kf == ke && f < e);
+        }
+        st->order[rk] = e;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&st->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int i = 0; i < N; ++i) { st->tstart[i] = acc; acc += st->ntile[st->order[i]]; }
+        st->tstart[N] = acc;
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                 // both CTAs' barriers exist before any remote arrive or TMA completion
+    tc_fence_after();
+    const uint32_t tmem_base = st->tmem_base;
+    const int total_tiles = st->tstart[N];
+    volatile int *abort_flag = &st->abort_flag;
+
+    if (warp == 0) {
+        // ===================== TMA producer (both CTAs) =====================
+        if (lane == 0) {
+            int stage = 0, cursor = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+                const Tile t = decode_tile2<KIND>(prm, st, tile, cursor, rank);
+                const uint32_t bytes = (uint32_t)(t.a_boxes + t.a_boxes_peer + 2 * t.b_boxes) * kBoxBytes;
+                for (int kb = 0; kb < t.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+                    const uint32_t leader_bar = map_to_cta(smem_u32(&st->full[stage]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&st->full[stage]), bytes);
+                    const uint32_t a_dst = stage_base + stage * kStageBytes2;
+                    issue_loads2<KIND>(maps, t, rank, kb, a_dst, a_dst + kARegion2, leader_bar);
+                    ++issued;
+                    if (++stage == kStages2) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok && rank == 0) {
+                const int n = issued < kStages2 ? (int)issued : kStages2;
+                for (int i = 1; i <= n; ++i) {
+                    int s = stage - i;
+                    uint32_t ph = phase;
+                    if (s < 0) { s += kStages2; ph ^= 1u; }
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(smem_u32(&st->full[s]), ph) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===================== MMA issuer (leader CTA only) =====================
+        if (lane == 0 && rank == 0) {
+            int stage = 0, cursor = 0, it = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            constexpr bool a_mn = KindTraits<KIND>::a_mn, b_mn = KindTraits<KIND>::b_mn;
+            constexpr uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
+            constexpr uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+            for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
+                const Tile t = decode_tile2<KIND>(prm, st, tile, cursor, 0);
+                const int acc = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + (uint32_t)(acc * kAccCols);
+                const uint32_t idesc = make_idesc_pair(a_mn, b_mn, t.n_mma);
+                for (int kb = 0; kb < t.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->full[stage]), phase, abort_flag, prm.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stage_base + stage * kStageBytes2;
+                    const uint64_t adesc = make_desc(a_addr, a_mn);
+                    const uint64_t bdesc = make_desc(a_addr + kARegion2, b_mn);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_bf16_pair(tacc, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
+                                       (kb > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit_pair(smem_u32(&st->empty[stage]));
+                    if (++stage == kStages2) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (t.nk > 0) {
+                    umma_commit_pair(smem_u32(&st->tmem_full[acc]));
+                } else {
+                    mbar_arrive(smem_u32(&st->tmem_full[acc]));
+                    mbar_arrive_cluster(map_to_cta(smem_u32(&st->tmem_full[acc]), 1));
+                }
+            }
+        }
+    } else {
+        // ===================== epilogue (warps 2..9, both CTAs) =====================
+        const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int row = quad * 32 + lane;
+        int cursor = 0, it = 0;
+        bool ok = true;
+        for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++it) {
+            const Tile t = decode_tile2<KIND>(prm, st, tile, cursor, rank);
+            const int acc = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, prm.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
+            if (t.mrows > 0) {
+                // split the accumulator columns between the two warps of a lane quadrant, store only valid ones
+                const int span = (KIND == TcUpGate) ? t.ncols : t.n_mma;
+                const int chalf = span >> 1;
+                const int c0 = half * chalf, c1 = min((half + 1) * chalf, t.ncols);
+                if (c0 < c1) epilogue_row<KIND>(prm, t, tacc, row, c0, c1);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (rank == 0) mbar_arrive(smem_u32(&st->tmem_empty[acc]));
+                else mbar_arrive_cluster(map_to_cta(smem_u32(&st->tmem_empty[acc]), 0));
+            }
+        }
+    }
+
+    // ---- teardown: nobody leaves while its partner may still touch its shared or tensor memory ----
+    tc_fence_before();
+    __syncthreads();
+    __syncwarp();
+    cluster_sync_all();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
 // ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
@@ -717,9 +1076,45 @@ TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *
     return prm;
 }
 
+// Launches the two-CTA kernel with as many clusters as can be resident at once (tiles are dealt
+// statically, so a cluster that is not resident would hold its share back).
+template <int KIND>
+cudaError_t launch_kind_pair(const TcMaps &maps, const TcParams &prm, int sms, cudaStream_t s, int *launches)
+{
+    auto kern = tc_grouped_gemm_pair<KIND>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes2);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(sms & ~1));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes2;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    static int max_clusters[6] = {0, 0, 0, 0, 0, 0};
+    if (max_clusters[KIND] == 0) {
+        int n = 0;
+        e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (e != cudaSuccess) return e;
+        if (n < 1) return cudaErrorInvalidConfiguration;
+        max_clusters[KIND] = n;
+    }
+    const int clusters = max_clusters[KIND] < sms / 2 ? max_clusters[KIND] : sms / 2;
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
+    e = cudaLaunchKernelEx(&cfg, kern, maps, prm);
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
 template <int KIND>
 cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
 {
+    if (g_pair_mask & (1 << KIND)) return launch_kind_pair<KIND>(maps, prm, grid, s, launches);
     auto kern = tc_grouped_gemm<KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;

@@ -17,6 +17,10 @@ struct TcPlan {
 bool tc_force_simt();
 void tc_set_force_simt(int on);
 
+// Which of the six products run on the two-CTA (cta_group::2) kernel: bit k = kind k.
+void tc_set_pair_mask(int mask);
+int tc_pair_mask();
+
 // The six grouped products of the layer (Sec. 3.1, Eq. 4 and its gradient).
 enum TcKind : int {
     TcUpGate = 0,       // Hm = g * silu(xp Wg^T) * (xp Wu^T), optionally saving B*silu'(A) and silu(A)

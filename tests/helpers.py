@@ -2,6 +2,8 @@
 Python binding and the fp64 oracle on the same seeded inputs."""
 from __future__ import annotations
 
+import os
+
 import numpy as np
 
 from oracle import modse_oracle as O
@@ -55,6 +57,8 @@ def run_gpu(inp: I.LayerInputs, backward: bool, save: bool | None = None, out_f3
     cfg = inp.cfg
     dt = torch.float32 if cfg.dtype == "f32" else torch.bfloat16
     dev = "cuda"
+    if "MODSE_TEST_PAIR_MASK" in os.environ:           # run the suite against the two-SM kernels
+        B.debug_set_pair_kernels(int(os.environ["MODSE_TEST_PAIR_MASK"]))
     layer = B.ModseLayer(cfg.d_model, cfg.ffn_sizes, cfg.top_k)
     layer.set_output_f32(out_f32)
     odt = torch.float32 if out_f32 else dt
@@ -97,7 +101,7 @@ def run_oracle(inp: I.LayerInputs, backward: bool):
     return out
 
 
-def check_routing(gpu_rt, rt, gate_tol=1e-6):
+def check_routing(gpu_rt, rt, gate_tol=5e-6):
     for name in ("topk_idx", "counts", "counts_slot", "offsets", "row_of", "token_of"):
         np.testing.assert_array_equal(gpu_rt[name], getattr(rt, name), err_msg=name)
     assert np.max(np.abs(gpu_rt["topk_gate"] - rt.topk_gate)) <= gate_tol

@@ -1,7 +1,8 @@
 """GPU parity: the CUDA library through its C ABI against the fp64 oracle,
 element by element, at sizes the oracle finishes in seconds.
 
-Tolerances: routing tables bit-exact, gates 1e-6 absolute, every floating
+Tolerances: routing tables bit-exact, gates 5e-6 absolute (fp32 logits summed over up to
+2048 products on tensor cores: measured 1.4e-6 at d = 2048), every floating
 tensor max|err|/RMS(ref) <= 1e-4 for the fp32 type and <= 2e-2 for bf16."""
 import dataclasses
 
