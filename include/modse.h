@@ -158,6 +158,36 @@ int modse_last_launch_count(const modse_layer_t *layer);
  * accumulation over micro-batches in fp32.  No effect on fp32 layers.        */
 modse_status_t modse_set_output_f32(modse_layer_t *layer, int on);
 
+/* Routing only, with no device allocation by anyone.  (The paper has no
+ * counterpart: this is a packaging variant of the router stage of Eq. 2-3.)
+ *
+ * For callers that cannot allocate device memory - a plugin invoked from a
+ * framework callback where cudaMalloc is off limits because it synchronises
+ * the device and can fail mid-step, code living inside a memory pool it does
+ * not own, or a tool that only wants the routing tables - the scratch of the
+ * router and rank kernels lives in a fixed 4 MiB array inside the library
+ * (every GPU that loads the library holds it until the process exits).  The
+ * caller passes only inputs and outputs, all device pointers:
+ *   x [T,d], w_router [N,d]  in `dtype`, 16-byte aligned
+ *   topk_idx [T,k] int32, topk_gate [T,k] fp32, counts [N], counts_slot [k,N],
+ *   offsets [N+1], row_of [T,k], token_of [k*T]  - same meaning and the same
+ *   values as modse_get_routing after modse_forward.
+ * Limits: the scratch must fit the array - about 4*k*T*3 + 1016*N bytes plus
+ * k*N*4 bytes per 64 tokens, e.g. T <= 100000 tokens for 8 experts, top-2;
+ * larger batches return MODSE_ERR_WORKSPACE_TOO_SMALL (nothing is launched).
+ * modse_route_static_scratch_capacity() returns the array size in bytes.
+ * The first call on each device looks up the array's device address (a host
+ * call, no allocation); make that first call before any stream capture.
+ * All calls share the one array and it keeps the last call's contents (the
+ * call clears what must start at zero): two calls that overlap on the GPU -
+ * different streams, or different host threads - race on it; serialise them.
+ * Calls no cudaMalloc/cudaFree and no allocating library routine.            */
+modse_status_t modse_route_static_scratch(modse_dtype_t dtype, int d_model, int n_experts, int top_k,
+                                          const void *x, const void *w_router, int n_tokens, int *topk_idx,
+                                          float *topk_gate, int *counts, int *counts_slot, int *offsets,
+                                          int *row_of, int *token_of, void *cuda_stream);
+size_t modse_route_static_scratch_capacity(void);
+
 /* Per-stage device timing (profiling aid).  After modse_stage_timing_begin the
  * next max_calls forward/backward calls on this layer bracket each of their
  * stages with a pair of CUDA events on the call's stream (no work is skipped

@@ -84,6 +84,9 @@ def load():
     lib.modse_check_device_status.argtypes = [vp, vp, vp]
     lib.modse_last_launch_count.restype = ci
     lib.modse_last_launch_count.argtypes = [vp]
+    lib.modse_route_static_scratch.restype = ci
+    lib.modse_route_static_scratch.argtypes = [ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.modse_route_static_scratch_capacity.restype = sz
     lib.modse_set_output_f32.restype = ci
     lib.modse_set_output_f32.argtypes = [vp, ci]
     lib.modse_stage_timing_begin.restype = ci
@@ -102,6 +105,33 @@ def load():
 
 def status_string(status: int) -> str:
     return load().modse_status_string(int(status)).decode()
+
+
+def route_static_scratch(x, w_router, top_k: int):
+    """Routing tables of a batch through modse_route_static_scratch: no workspace, the
+    library's built-in scratch array is used.  Returns a dict of freshly created output
+    tensors (the outputs are the caller's; only the scratch is the library's)."""
+    import torch
+    T, d = x.shape
+    N = w_router.shape[0]
+    dev = x.device
+    out = {
+        "topk_idx": torch.empty((T, top_k), dtype=torch.int32, device=dev),
+        "topk_gate": torch.empty((T, top_k), dtype=torch.float32, device=dev),
+        "counts": torch.empty(N, dtype=torch.int32, device=dev),
+        "counts_slot": torch.empty((top_k, N), dtype=torch.int32, device=dev),
+        "offsets": torch.empty(N + 1, dtype=torch.int32, device=dev),
+        "row_of": torch.empty((T, top_k), dtype=torch.int32, device=dev),
+        "token_of": torch.empty(T * top_k, dtype=torch.int32, device=dev),
+    }
+    st = load().modse_route_static_scratch(
+        _dtype_code(x), d, N, top_k, x.data_ptr(), w_router.data_ptr(), T, out["topk_idx"].data_ptr(),
+        out["topk_gate"].data_ptr(), out["counts"].data_ptr(), out["counts_slot"].data_ptr(),
+        out["offsets"].data_ptr(), out["row_of"].data_ptr(), out["token_of"].data_ptr(),
+        ctypes.c_void_p(torch.cuda.current_stream().cuda_stream))
+    if st != MODSE_OK:
+        raise ModseError(st, "modse_route_static_scratch")
+    return out
 
 
 def stage_name(i: int) -> str:
