@@ -208,11 +208,13 @@ const char *modse_stage_name(int stage);
  * be called with save_for_backward = 1.  Off by default.                    */
 void modse_debug_use_fma_path(int on);
 
-/* Tuning aid, process-wide: bit k of `mask` selects, for grouped product k
+/* Tuning aid, process-wide: which of three tile shapes each grouped product k
  * (0 up/gate, 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate dgrad, 5 up/gate
- * wgrad), the kernel that computes 256-row tiles on pairs of SMs instead of
- * 128-row tiles on single SMs.  Results are the same up to fp32 summation
- * order inside the tensor cores.                                            */
+ * wgrad) runs on.  Bit k of `mask`: 256-row tiles on pairs of SMs
+ * (cta_group::2); bit 8+k: 256-row tiles on one SM (two accumulators sharing
+ * the column operand); neither: 128-row tiles on one SM.  The library's default
+ * is bits 8+{1,3,4,5}.  Every choice gives bit-identical results (the order
+ * in which each output element is summed does not depend on the tile shape). */
 void modse_debug_set_pair_kernels(int mask);
 
 #ifdef __cplusplus

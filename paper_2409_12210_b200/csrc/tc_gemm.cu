@@ -49,8 +49,12 @@ namespace modse {
 
 static int g_force_simt = 0;
 static int g_pair_mask = 0;      // bit k: product kind k runs on the two-CTA kernel
-void tc_set_pair_mask(int mask) { g_pair_mask = mask & 63; }
-int tc_pair_mask() { return g_pair_mask; }
+// bit k: product kind k runs on the 256-row single-CTA kernel.  Default: the four products with long
+// K loops (down, down wgrad, up/gate dgrad, up/gate wgrad), where it measured 4-13 % faster than the
+// 128-row kernel; the two products with K = d and heavy epilogues (up/gate, down dgrad) measured slower.
+static int g_wide_mask = (1 << 1) | (1 << 3) | (1 << 4) | (1 << 5);
+void tc_set_pair_mask(int mask) { g_pair_mask = mask & 63; g_wide_mask = (mask >> 8) & 63; }
+int tc_pair_mask() { return g_pair_mask | (g_wide_mask << 8); }
 
 bool tc_force_simt() { return g_force_simt != 0; }
 void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
@@ -991,6 +995,324 @@ tc_grouped_gemm_pair(const __grid_constant__ TcMaps maps, const __grid_constant_
     }
 }
 
+// ===========================================================================
+// Wide variant: one CTA computes a 256-row tile as two 128-row halves that
+// share the column operand.  A k-block then stages 32 KB of rows + 32 KB of
+// columns for twice the MMA work of the 128-row kernel, i.e. 2/3 of the bytes
+// per FLOP through L2 -> shared memory, which is what bounds the 128-row
+// kernel (it needs ~19.5 TB/s of L2 reads at the MMA rate; the path saturates
+// near 22 TB/s).  The price: both accumulators (2 x 256 TMEM columns) belong
+// to the current tile, so the epilogue of a tile overlaps only the part of the
+// next tile's main loop that does not touch the half being drained.  Used for
+// the products with long K loops, where that exposure is a few percent.
+// ===========================================================================
+constexpr int kStagesW = 3;
+constexpr int kARegionW = 4 * kBoxBytes;            // two halves of 128 rows x 64 K
+constexpr int kStageBytesW = kARegionW + kBRegion;  // 64 KB
+struct SmemTailW {
+    unsigned long long full[kStagesW], empty[kStagesW], tmem_full[1], tmem_empty[2];
+    unsigned int tmem_base;
+    int abort_flag;
+    int order[kMaxExperts];
+    int key[kMaxExperts];
+    int ntile[kMaxExperts];
+    int tstart[kMaxExperts + 1];
+};
+constexpr size_t kSmemBytesW = 1024 + (size_t)kStagesW * kStageBytesW + sizeof(SmemTailW);
+
+template <int KIND>
+__device__ __forceinline__ void expert_shape_wide(int cp, int h, int d, int &mt, int &nt, int &nk)
+{
+    if constexpr (KIND == TcUpGate)      { mt = (cp + 255) / 256; nt = (h + 127) / 128; nk = d / 64; }
+    if constexpr (KIND == TcDown)        { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = h / 64; }
+    if constexpr (KIND == TcDownDgrad)   { mt = (cp + 255) / 256; nt = (h + 255) / 256; nk = d / 64; }
+    if constexpr (KIND == TcDownWgrad)   { mt = (d + 255) / 256;  nt = (h + 255) / 256; nk = cp / 64; }
+    if constexpr (KIND == TcUpGateDgrad) { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = 2 * (h / 64); }
+    if constexpr (KIND == TcUpGateWgrad) { mt = 2 * ((h + 255) / 256); nt = (d + 255) / 256; nk = cp / 64; }
+}
+
+// First half (rows m0 .. m0+127) of wide tile `tile`; a_boxes_peer carries the second half's boxes.
+template <int KIND>
+__device__ __forceinline__ Tile decode_tile_wide(const TcParams &prm, const SmemTailW *st, int tile, int &cursor)
+{
+    const int N = prm.meta.N, d = prm.meta.d;
+    while (cursor + 1 < N && tile >= st->tstart[cursor + 1]) ++cursor;
+    Tile t;
+    t.e = st->order[cursor];
+    t.ho = prm.meta.hoff[t.e];
+    t.h = prm.meta.hoff[t.e + 1] - t.ho;
+    t.prow0 = prm.poffsets[t.e];
+    t.cp = prm.poffsets[t.e + 1] - t.prow0;
+    t.pbase = (int)(prm.ebase[t.e] >> 6);
+    int mt, nt, nk;
+    expert_shape_wide<KIND>(t.cp, t.h, d, mt, nt, nk);
+    const int local = tile - st->tstart[cursor];
+    constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
+    int mb = n_fastest ? local / nt : local % mt;
+    const int nb = n_fastest ? local % nt : local / mt;
+    t.nk = nk;
+    t.which = 0;
+    int row_extent;
+    if constexpr (KIND == TcDownWgrad) row_extent = d;
+    else if constexpr (KIND == TcUpGateWgrad) { row_extent = t.h; t.which = mb & 1; mb >>= 1; }
+    else row_extent = t.cp;
+    t.m0 = mb * 256;
+    t.mrows = max(0, min(128, row_extent - t.m0));
+    t.a_boxes = t.mrows / 64;
+    t.a_boxes_peer = max(0, min(128, row_extent - t.m0 - 128)) / 64;
+    t.b_off = 0;
+    if constexpr (KIND == TcUpGate) {
+        t.n0 = nb * 128; t.ncols = min(128, t.h - t.n0);
+        t.n_mma = 2 * t.ncols; t.b_boxes = t.n_mma / 64;
+    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad) {
+        t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
+        t.n_mma = t.ncols; t.b_boxes = t.ncols / 64;
+    } else {
+        t.n0 = nb * 256; t.ncols = min(256, t.h - t.n0);
+        t.n_mma = t.ncols; t.b_boxes = t.ncols / 64;
+    }
+    return t;
+}
+
+__device__ __forceinline__ Tile second_half(const Tile &t)
+{
+    Tile u = t;
+    u.m0 = t.m0 + 128;
+    u.a_boxes = t.a_boxes_peer;
+    u.mrows = 64 * t.a_boxes_peer;
+    return u;
+}
+
+// Row-operand boxes of one 128-row half.
+template <int KIND>
+__device__ __forceinline__ void load_rows(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
+{
+    if constexpr (KIND == TcUpGate) {
+        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.xp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+    } else if constexpr (KIND == TcDown) {
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d(dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + kb * t.cp + t.m0 + 64 * i);
+    } else if constexpr (KIND == TcDownDgrad) {
+        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.dyp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+    } else if constexpr (KIND == TcDownWgrad) {
+        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
+    } else if constexpr (KIND == TcUpGateDgrad) {
+        const int half = t.h / 64;
+        const bool second = kb >= half;
+        const int kk = second ? kb - half : kb;
+        const CUtensorMap *am = second ? &maps.db : &maps.da;
+        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, am, bar, 0, t.pbase + kk * t.cp + t.m0 + 64 * i);
+    } else {
+        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d(dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
+    }
+}
+
+// Column-operand boxes of a tile.
+template <int KIND>
+__device__ __forceinline__ void load_cols(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
+{
+    if constexpr (KIND == TcUpGate) {
+        const int nb = t.ncols / 64;
+        for (int i = 0; i < nb; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wgate, bar, kb * 64, t.ho + t.n0 + 64 * i);
+        for (int i = 0; i < nb; ++i) tma_load_2d(dst + (nb + i) * kBoxBytes, &maps.wup, bar, kb * 64, t.ho + t.n0 + 64 * i);
+    } else if constexpr (KIND == TcDown) {
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wdown, bar, t.ho + kb * 64, t.n0 + 64 * i);
+    } else if constexpr (KIND == TcDownDgrad) {
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + 64 * i, kb * 64);
+    } else if constexpr (KIND == TcDownWgrad) {
+        for (int i = 0; i < t.b_boxes; ++i)
+            tma_load_2d(dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + (t.n0 / 64 + i) * t.cp + kb * 64);
+    } else if constexpr (KIND == TcUpGateDgrad) {
+        const int half = t.h / 64;
+        const bool second = kb >= half;
+        const int kk = second ? kb - half : kb;
+        const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, bm, bar, t.n0 + 64 * i, t.ho + kk * 64);
+    } else {
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.xp, bar, t.n0 + 64 * i, t.prow0 + kb * 64);
+    }
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_grouped_gemm_wide(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
+    unsigned char *smem = smem_raw + pad;
+    const uint32_t stage_base = raw + pad;
+    SmemTailW *st = reinterpret_cast<SmemTailW *>(smem + (size_t)kStagesW * kStageBytesW);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int N = prm.meta.N, d = prm.meta.d;
+
+    for (int e = tid; e < N; e += kThreads) {
+        const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
+        const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
+        int mt, nt, nk;
+        expert_shape_wide<KIND>(cp, h, d, mt, nt, nk);
+        st->ntile[e] = mt * nt;
+        st->key[e] = nk;
+    }
+    if (tid == 0) {
+        for (int s = 0; s < kStagesW; ++s) {
+            mbar_init(smem_u32(&st->full[s]), 1);
+            mbar_init(smem_u32(&st->empty[s]), 1);
+        }
+        mbar_init(smem_u32(&st->tmem_full[0]), 1);
+        mbar_init(smem_u32(&st->tmem_empty[0]), 256);
+        mbar_init(smem_u32(&st->tmem_empty[1]), 256);
+        st->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    for (int e = tid; e < N; e += kThreads) {
+        int rk = 0;
+        const int ke = st->key[e];
+        for (int f = 0; f < N; ++f) {
+            const int kf = st->key[f];
+            rk += (kf > ke) || (kf == ke && f < e);
+        }
+        st->order[rk] = e;
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&st->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int i = 0; i < N; ++i) { st->tstart[i] = acc; acc += st->ntile[st->order[i]]; }
+        st->tstart[N] = acc;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = st->tmem_base;
+    const int total_tiles = st->tstart[N];
+    volatile int *abort_flag = &st->abort_flag;
+
+    if (warp == 0) {
+        // ===================== TMA producer =====================
+        if (lane == 0) {
+            int stage = 0, cursor = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const Tile t0 = decode_tile_wide<KIND>(prm, st, tile, cursor);
+                const Tile t1 = second_half(t0);
+                const uint32_t bytes = (uint32_t)(t0.a_boxes + t1.a_boxes + t0.b_boxes) * kBoxBytes;
+                for (int kb = 0; kb < t0.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(&st->full[stage]);
+                    mbar_arrive_expect_tx(bar, bytes);
+                    const uint32_t a_dst = stage_base + stage * kStageBytesW;
+                    load_rows<KIND>(maps, t0, kb, a_dst, bar);
+                    load_rows<KIND>(maps, t1, kb, a_dst + kARegion, bar);
+                    load_cols<KIND>(maps, t0, kb, a_dst + kARegionW, bar);
+                    ++issued;
+                    if (++stage == kStagesW) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                const int n = issued < kStagesW ? (int)issued : kStagesW;
+                for (int i = 1; i <= n; ++i) {
+                    int s = stage - i;
+                    uint32_t ph = phase;
+                    if (s < 0) { s += kStagesW; ph ^= 1u; }
+                    const unsigned long long tb = global_ns();
+                    while (!mbar_try_wait(smem_u32(&st->full[s]), ph) && global_ns() - tb < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===================== MMA issuer =====================
+        if (lane == 0) {
+            int stage = 0, cursor = 0;
+            uint32_t phase = 0;
+            uint32_t use0 = 0, use1 = 0;         // how often each accumulator has been handed to the epilogue
+            bool ok = true;
+            constexpr bool a_mn = KindTraits<KIND>::a_mn, b_mn = KindTraits<KIND>::b_mn;
+            constexpr uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
+            constexpr uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const Tile t = decode_tile_wide<KIND>(prm, st, tile, cursor);
+                const bool two = t.a_boxes_peer > 0;
+                if (!mbar_wait(smem_u32(&st->tmem_empty[0]), (use0 & 1u) ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t idesc = make_idesc(a_mn, b_mn, t.n_mma);
+                for (int kb = 0; kb < t.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->full[stage]), phase, abort_flag, prm.status)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stage_base + stage * kStageBytesW;
+                    const uint64_t adesc0 = make_desc(a_addr, a_mn);
+                    const uint64_t adesc1 = make_desc(a_addr + kARegion, a_mn);
+                    const uint64_t bdesc = make_desc(a_addr + kARegionW, b_mn);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_bf16(tmem_base, adesc0 + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
+                                  (kb > 0 || ks > 0) ? 1u : 0u);
+                    if (two) {
+                        if (kb == 0) {
+                            // the second accumulator may still be draining: the first half's MMAs above are already queued
+                            if (!mbar_wait(smem_u32(&st->tmem_empty[1]), (use1 & 1u) ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+                            tc_fence_after();
+                        }
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_bf16(tmem_base + kAccCols, adesc1 + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step),
+                                      idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&st->empty[stage]));
+                    if (++stage == kStagesW) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (t.nk > 0) umma_commit(smem_u32(&st->tmem_full[0]));
+                else mbar_arrive(smem_u32(&st->tmem_full[0]));
+                ++use0;
+                if (two) ++use1;
+            }
+        }
+    } else {
+        // ===================== epilogue (warps 2..9) =====================
+        const int quad = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int row = quad * 32 + lane;
+        int cursor = 0, it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++it) {
+            const Tile t0 = decode_tile_wide<KIND>(prm, st, tile, cursor);
+            if (!mbar_wait(smem_u32(&st->tmem_full[0]), (uint32_t)it & 1u, abort_flag, prm.status)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16);
+            const int chalf = t0.ncols >> 1;
+            epilogue_row<KIND>(prm, t0, tacc, row, half * chalf, (half + 1) * chalf);
+            tc_fence_before();
+            mbar_arrive(smem_u32(&st->tmem_empty[0]));
+            if (t0.a_boxes_peer > 0) {
+                const Tile t1 = second_half(t0);
+                epilogue_row<KIND>(prm, t1, tacc + kAccCols, row, half * chalf, (half + 1) * chalf);
+                tc_fence_before();
+                mbar_arrive(smem_u32(&st->tmem_empty[1]));
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
 // ---------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------
@@ -1112,8 +1434,21 @@ cudaError_t launch_kind_pair(const TcMaps &maps, const TcParams &prm, int sms, c
 }
 
 template <int KIND>
+cudaError_t launch_kind_wide(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
+{
+    auto kern = tc_grouped_gemm_wide<KIND>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytesW);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, kSmemBytesW, s>>>(maps, prm);
+    e = cudaGetLastError();
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+template <int KIND>
 cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
 {
+    if (g_wide_mask & (1 << KIND)) return launch_kind_wide<KIND>(maps, prm, grid, s, launches);
     if (g_pair_mask & (1 << KIND)) return launch_kind_pair<KIND>(maps, prm, grid, s, launches);
     auto kern = tc_grouped_gemm<KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
