@@ -232,11 +232,13 @@ def main():
     do_bwd = cfg.backward
     ws = layer.alloc_workspace(dt, T, do_bwd, dev)
 
-    def step():
-        layer.forward(wr, wg, wu, wd, x, y, ws, do_bwd)
+    def step(xb=None, dyb=None, yb=None, dxb=None):
+        xb, dyb = (x if xb is None else xb), (dy if dyb is None else dyb)
+        yb, dxb = (y if yb is None else yb), (dx if dxb is None else dxb)
+        layer.forward(wr, wg, wu, wd, xb, yb, ws, do_bwd)
         n = layer.last_launch_count()
         if do_bwd:
-            layer.backward(wr, wg, wu, wd, x, dy, dx, dwr, dwg, dwu, dwd, ws)
+            layer.backward(wr, wg, wu, wd, xb, dyb, dxb, dwr, dwg, dwu, dwd, ws)
             n += layer.last_launch_count()
         return n
 
@@ -279,21 +281,48 @@ def main():
     h2d = hx.numel() * hx.element_size() * (2 if do_bwd else 1)
     d2h = hy.numel() * hy.element_size() * (2 if do_bwd else 1)
 
-    def e2e_step():
-        x.copy_(hx, non_blocking=True)
-        if do_bwd:
-            dy.copy_(hdy, non_blocking=True)
-        step()
-        hy.copy_(y, non_blocking=True)
-        if do_bwd:
-            hdx.copy_(dx, non_blocking=True)
+    # Every step copies its inputs host -> device and its results device -> host; the copies of
+    # neighbouring steps run on their own streams (two device buffers each way), as a data loader
+    # that prefetches the next batch would.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    xin, dyin = [torch.empty_like(x) for _ in range(2)], [torch.empty_like(x) for _ in range(2)]
+    yout, dxout = [torch.empty_like(x) for _ in range(2)], [torch.empty_like(x) for _ in range(2)]
+    E = lambda: [torch.cuda.Event() for _ in range(2)]
+    ev_in, ev_done, ev_out = E(), E(), E()
 
-    for _ in range(3):
-        e2e_step()
+    def load(b, first):
+        with torch.cuda.stream(s_in):
+            if not first:
+                s_in.wait_event(ev_done[b])          # the step that last read this buffer pair is over
+            xin[b].copy_(hx, non_blocking=True)
+            if do_bwd:
+                dyin[b].copy_(hdy, non_blocking=True)
+            ev_in[b].record(s_in)
+
+    def e2e_run(n_steps):
+        comp = torch.cuda.current_stream()
+        load(0, True)
+        for i in range(n_steps):
+            b = i & 1
+            if i + 1 < n_steps:
+                load((i + 1) & 1, i < 1)
+            comp.wait_event(ev_in[b])
+            if i >= 2:
+                comp.wait_event(ev_out[b])           # results of step i-2 have left this buffer pair
+            step(xin[b], dyin[b], yout[b], dxout[b])
+            ev_done[b].record(comp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[b])
+                hy.copy_(yout[b], non_blocking=True)
+                if do_bwd:
+                    hdx.copy_(dxout[b], non_blocking=True)
+                ev_out[b].record(s_out)
+        comp.wait_stream(s_out)
+
+    e2e_run(3)
     sync_all()
     ev0.record()
-    for _ in range(K):
-        e2e_step()
+    e2e_run(K)
     ev1.record()
     sync_all()
     ms_e2e = ev0.elapsed_time(ev1)

@@ -171,7 +171,8 @@ router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok,
 
 // ---------------------------------------------------------------------------
 // Router, bf16 with at most 16 experts: the logits of 16 tokens per warp come
-// from mma.sync m16n8k16 (bf16 x bf16 -> fp32) fed straight from global memory.
+// from mma.sync m16n8k16 (bf16 x bf16 -> fp32) fed straight from global memory
+// (two warps per 16 tokens, each summing half of the k range, added in fp32).
 // A lane loads 8 consecutive elements (16 bytes) of two token rows and of one
 // router row per k-chunk of 32 and uses them as the operands of two MMAs: the
 // sum over k does not depend on which k index sits in which operand slot as
@@ -197,19 +198,21 @@ __device__ __forceinline__ void quad_argmax(float &bv, int &bi)
 }
 
 template <int NT>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256)
 router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w_router, int Ttok, int d,
                   int N, int k, int *__restrict__ topk_idx, float *__restrict__ topk_gate,
                   int *__restrict__ block_counts)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     int *cnt = reinterpret_cast<int *>(smem_raw);                                   // [k*N], padded to 128 bytes
-    __nv_bfloat16 *wsm = reinterpret_cast<__nv_bfloat16 *>(smem_raw + 128);         // [NT*8][d + 8]
+    float *part = reinterpret_cast<float *>(smem_raw + 128);                        // [4 groups][32 lanes][NT*4]
+    __nv_bfloat16 *wsm = reinterpret_cast<__nv_bfloat16 *>(smem_raw + 128 + 4 * 32 * NT * 4 * sizeof(float));
     const int ldw = d + 8;                                                          // 16-byte skew: conflict-free rows
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, tq = lane & 3;
-    for (int i = tid; i < k * N; i += 128) cnt[i] = 0;
-    for (int i = tid * 8; i < NT * 8 * d; i += 128 * 8) {
+    const int grp = warp & 3, khalf = warp >> 2;        // 16-token group; which half of the k range
+    for (int i = tid; i < k * N; i += 256) cnt[i] = 0;
+    for (int i = tid * 8; i < NT * 8 * d; i += 256 * 8) {
         const int r = i / d, c = i % d;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (r < N) v = *reinterpret_cast<const uint4 *>(w_router + (size_t)r * d + c);
@@ -217,7 +220,7 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
     }
     __syncthreads();
 
-    const int t0 = blockIdx.x * kRouterTokB + warp * 16;
+    const int t0 = blockIdx.x * kRouterTokB + grp * 16;
     const int r0 = t0 + g, r1 = t0 + g + 8;
     const bool v0 = r0 < Ttok, v1 = r1 < Ttok;
     const uint4 *x0 = reinterpret_cast<const uint4 *>(x + (size_t)(v0 ? r0 : 0) * d + tq * 8);
@@ -225,10 +228,11 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-#pragma unroll 4
-    for (int c0 = 0; c0 < d; c0 += 32) {
+    const int cbeg = khalf * (d >> 1), cend = cbeg + (d >> 1);
+#pragma unroll 8
+    for (int c0 = cbeg; c0 < cend; c0 += 32) {
         const uint4 za = make_uint4(0u, 0u, 0u, 0u);
-        const uint4 xa = v0 ? x0[c0 >> 3] : za;     // 32 elements = 4 uint4 per row chunk; this lane's is index c0/8 + (tq folded into base)
+        const uint4 xa = v0 ? x0[c0 >> 3] : za;
         const uint4 xb = v1 ? x1[c0 >> 3] : za;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
@@ -237,47 +241,64 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
             mma_bf16_16816(acc[nt], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
         }
     }
-    // acc[nt][0..1]: token r0, experts nt*8 + 2tq, +1;  acc[nt][2..3]: token r1, same experts
+    // second-half warps hand their partial logits to the first-half warp of the same token group
+    if (khalf == 1) {
 #pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        const int t = half ? r1 : r0;
-        float zsel[2] = {0.f, 0.f};
-        int isel[2] = {kNoIndex, kNoIndex};
-        for (int j = 0; j < k; ++j) {
-            float bv = -INFINITY;
-            int bi = kNoIndex;
+        for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
+            for (int u = 0; u < 4; ++u) part[((grp * 32 + lane) * NT + nt) * 4 + u] = acc[nt][u];
+    }
+    __syncthreads();
+    if (khalf == 0) {
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int e = nt * 8 + 2 * tq + u;
-                    const float v = acc[nt][2 * half + u];
-                    const bool usable = e < N && !(j > 0 && e == isel[0]);
-                    if (usable && (bi == kNoIndex || v > bv)) { bv = v; bi = e; }
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int u = 0; u < 4; ++u) acc[nt][u] += part[((grp * 32 + lane) * NT + nt) * 4 + u];
+        // acc[nt][0..1]: token r0, experts nt*8 + 2tq, +1;  acc[nt][2..3]: token r1, same experts
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int t = half ? r1 : r0;
+            float zsel[2] = {0.f, 0.f};
+            int isel[2] = {kNoIndex, kNoIndex};
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                if (j < k) {
+                    float bv = -INFINITY;
+                    int bi = kNoIndex;
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int e = nt * 8 + 2 * tq + u;
+                            const float v = acc[nt][2 * half + u];
+                            const bool usable = e < N && !(j > 0 && e == isel[0]);
+                            if (usable && (bi == kNoIndex || v > bv)) { bv = v; bi = e; }
+                        }
+                    quad_argmax(bv, bi);
+                    zsel[j] = bv;
+                    isel[j] = bi;
                 }
-            quad_argmax(bv, bi);
-            zsel[j] = bv;
-            isel[j] = bi;
-        }
-        if (tq == 0 && t < Ttok) {
-            if (k == 1) {
-                topk_idx[t] = isel[0];
-                topk_gate[t] = 1.0f;
-                atomicAdd(&cnt[isel[0]], 1);
-            } else {
-                const float w1 = expf(zsel[1] - zsel[0]);
-                const float den = 1.0f + w1;
-                topk_idx[2 * (size_t)t] = isel[0];
-                topk_idx[2 * (size_t)t + 1] = isel[1];
-                topk_gate[2 * (size_t)t] = 1.0f / den;
-                topk_gate[2 * (size_t)t + 1] = w1 / den;
-                atomicAdd(&cnt[isel[0]], 1);
-                atomicAdd(&cnt[N + isel[1]], 1);
+            }
+            if (tq == 0 && t < Ttok) {
+                if (k == 1) {
+                    topk_idx[t] = isel[0];
+                    topk_gate[t] = 1.0f;
+                    atomicAdd(&cnt[isel[0]], 1);
+                } else {
+                    const float w1 = expf(zsel[1] - zsel[0]);
+                    const float den = 1.0f + w1;
+                    topk_idx[2 * (size_t)t] = isel[0];
+                    topk_idx[2 * (size_t)t + 1] = isel[1];
+                    topk_gate[2 * (size_t)t] = 1.0f / den;
+                    topk_gate[2 * (size_t)t + 1] = w1 / den;
+                    atomicAdd(&cnt[isel[0]], 1);
+                    atomicAdd(&cnt[N + isel[1]], 1);
+                }
             }
         }
     }
     __syncthreads();
-    for (int i = tid; i < k * N; i += 128) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
+    for (int i = tid; i < k * N; i += 256) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
 }
 
 // ---------------------------------------------------------------------------
@@ -302,15 +323,33 @@ rank_kernel(LayerMeta m, int Ttok, int Pmax, int nblk, const int *__restrict__ b
     int *bidx = base + N;          // [64*k] this block's expert choices
 
     const int tid = threadIdx.x, b = blockIdx.x;
-    for (int p = tid; p < kN; p += 256) {
-        int before = 0, all = 0;
-        for (int bb = 0; bb < nblk; ++bb) {
-            const int c = block_counts[(size_t)bb * kN + p];
-            all += c;
-            if (bb < b) before += c;
+    // totals and "blocks before mine" sums per (slot, expert): the threads share the blocks of each
+    // pair and add their partial sums with integer shared-memory atomics (order does not matter)
+    for (int p = tid; p < 2 * kN; p += 256) tot[p] = 0;       // tot and pre are adjacent
+    __syncthreads();
+    {
+        const int groups = max(1, 256 / kN);
+        const int gidx = tid / kN, p = tid % kN;
+        if (gidx < groups && tid < 256) {
+            int before = 0, all = 0;
+            for (int bb = gidx; bb < nblk; bb += groups) {
+                const int c = block_counts[(size_t)bb * kN + p];
+                all += c;
+                if (bb < b) before += c;
+            }
+            atomicAdd(&tot[p], all);
+            atomicAdd(&pre[p], before);
         }
-        tot[p] = all;
-        pre[p] = before;
+        for (int q = 256 + tid; q < kN; q += 256) {            // more pairs than threads: the rest, one thread each
+            int before = 0, all = 0;
+            for (int bb = 0; bb < nblk; ++bb) {
+                const int c = block_counts[(size_t)bb * kN + q];
+                all += c;
+                if (bb < b) before += c;
+            }
+            tot[q] = all;
+            pre[q] = before;
+        }
     }
     const int t0 = b * kRouterTokB;
     for (int i = tid; i < kRouterTokB * k; i += 256) {
@@ -605,14 +644,14 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
                           const WsPtrs &p, cudaStream_t s, int *launches)
 {
     const int nblk = (T + kRouterTokB - 1) / kRouterTokB;
-    if (dt == MODSE_BF16 && m.N <= 16 && m.d % 32 == 0 && m.k * m.N * 4 <= 128) {
+    if (dt == MODSE_BF16 && m.N <= 16 && m.d % 64 == 0 && m.k * m.N * 4 <= 128) {
         const int nt = (m.N + 7) / 8;
-        const size_t smem = 128 + (size_t)nt * 8 * (m.d + 8) * 2;
+        const size_t smem = 128 + (size_t)4 * 32 * nt * 4 * sizeof(float) + (size_t)nt * 8 * (m.d + 8) * 2;
         if (smem <= 200 * 1024) {
             auto kern = nt == 1 ? router_mma_kernel<1> : router_mma_kernel<2>;
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            kern<<<nblk, 128, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
+            kern<<<nblk, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
                                          p.topk_idx, p.topk_gate, p.block_counts);
             MODSE_LAUNCH_CHECK();
             return cudaSuccess;
