@@ -172,7 +172,7 @@ router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok,
 // ---------------------------------------------------------------------------
 // Router, bf16 with at most 16 experts: the logits of 16 tokens per warp come
 // from mma.sync m16n8k16 (bf16 x bf16 -> fp32) fed straight from global memory
-// (two warps per 16 tokens, each summing half of the k range, added in fp32).
+// (four warps per 16 tokens, each summing a quarter of the k range, added in fp32).
 // A lane loads 8 consecutive elements (16 bytes) of two token rows and of one
 // router row per k-chunk of 32 and uses them as the operands of two MMAs: the
 // sum over k does not depend on which k index sits in which operand slot as
@@ -197,22 +197,26 @@ __device__ __forceinline__ void quad_argmax(float &bv, int &bi)
     }
 }
 
+constexpr int kRouterKSplit = 4;     // warps per 16-token group, each summing a quarter of the k range
+constexpr int kRouterMmaThreads = 4 * kRouterKSplit * 32;
+
 template <int NT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kRouterMmaThreads)
 router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w_router, int Ttok, int d,
                   int N, int k, int *__restrict__ topk_idx, float *__restrict__ topk_gate,
                   int *__restrict__ block_counts)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     int *cnt = reinterpret_cast<int *>(smem_raw);                                   // [k*N], padded to 128 bytes
-    float *part = reinterpret_cast<float *>(smem_raw + 128);                        // [4 groups][32 lanes][NT*4]
-    __nv_bfloat16 *wsm = reinterpret_cast<__nv_bfloat16 *>(smem_raw + 128 + 4 * 32 * NT * 4 * sizeof(float));
+    float *part = reinterpret_cast<float *>(smem_raw + 128);                        // [KS-1][4 groups][32 lanes][NT*4]
+    __nv_bfloat16 *wsm = reinterpret_cast<__nv_bfloat16 *>(smem_raw + 128 +
+                                                           (kRouterKSplit - 1) * 4 * 32 * NT * 4 * sizeof(float));
     const int ldw = d + 8;                                                          // 16-byte skew: conflict-free rows
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, tq = lane & 3;
-    const int grp = warp & 3, khalf = warp >> 2;        // 16-token group; which half of the k range
-    for (int i = tid; i < k * N; i += 256) cnt[i] = 0;
-    for (int i = tid * 8; i < NT * 8 * d; i += 256 * 8) {
+    const int grp = warp & 3, kpart = warp >> 2;        // 16-token group; which part of the k range
+    for (int i = tid; i < k * N; i += kRouterMmaThreads) cnt[i] = 0;
+    for (int i = tid * 8; i < NT * 8 * d; i += kRouterMmaThreads * 8) {
         const int r = i / d, c = i % d;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
         if (r < N) v = *reinterpret_cast<const uint4 *>(w_router + (size_t)r * d + c);
@@ -228,7 +232,7 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-    const int cbeg = khalf * (d >> 1), cend = cbeg + (d >> 1);
+    const int cbeg = kpart * (d / kRouterKSplit), cend = cbeg + d / kRouterKSplit;
 #pragma unroll 8
     for (int c0 = cbeg; c0 < cend; c0 += 32) {
         const uint4 za = make_uint4(0u, 0u, 0u, 0u);
@@ -241,19 +245,24 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
             mma_bf16_16816(acc[nt], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
         }
     }
-    // second-half warps hand their partial logits to the first-half warp of the same token group
-    if (khalf == 1) {
+    // the other warps hand their partial logits to the first warp of the same token group,
+    // which adds them in a fixed order
+    if (kpart > 0) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int u = 0; u < 4; ++u) part[((grp * 32 + lane) * NT + nt) * 4 + u] = acc[nt][u];
+            for (int u = 0; u < 4; ++u)
+                part[((((kpart - 1) * 4 + grp) * 32 + lane) * NT + nt) * 4 + u] = acc[nt][u];
     }
     __syncthreads();
-    if (khalf == 0) {
+    if (kpart == 0) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int q = 1; q < kRouterKSplit; ++q)
 #pragma unroll
-            for (int u = 0; u < 4; ++u) acc[nt][u] += part[((grp * 32 + lane) * NT + nt) * 4 + u];
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    acc[nt][u] += part[((((q - 1) * 4 + grp) * 32 + lane) * NT + nt) * 4 + u];
         // acc[nt][0..1]: token r0, experts nt*8 + 2tq, +1;  acc[nt][2..3]: token r1, same experts
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
@@ -298,7 +307,7 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
         }
     }
     __syncthreads();
-    for (int i = tid; i < k * N; i += 256) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
+    for (int i = tid; i < k * N; i += kRouterMmaThreads) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
 }
 
 // ---------------------------------------------------------------------------
@@ -578,12 +587,13 @@ __global__ void __launch_bounds__(256)
 router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int *__restrict__ topk_idx,
                   const float *__restrict__ dz, float *__restrict__ dwr_partial)
 {
+    constexpr int CPT = (sizeof(T) == 2) ? 2 : 1;        // columns per thread: one 4-byte load either way
     __shared__ float dzs[kRouterBwdTokB][8];
     __shared__ int idxs[kRouterBwdTokB][2];
     __shared__ float dzk[kRouterBwdTokB][2];
     const int tid = threadIdx.x;
     const int t0 = blockIdx.x * kRouterBwdTokB;
-    const int c = blockIdx.y * 256 + tid;
+    const int c = (blockIdx.y * 256 + tid) * CPT;
     const int ntok = min(kRouterBwdTokB, Ttok - t0);
     for (int i = tid; i < kRouterBwdTokB * 2; i += 256) {
         const int tl = i >> 1, j = i & 1;
@@ -602,18 +612,33 @@ router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const 
         }
         __syncthreads();
         if (c < d) {
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            float acc[8][CPT];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int u = 0; u < CPT; ++u) acc[i][u] = 0.f;
 #pragma unroll 8
             for (int tl = 0; tl < ntok; ++tl) {
-                float xv;
-                if (sizeof(T) == 4) xv = reinterpret_cast<const float *>(x)[(size_t)(t0 + tl) * d + c];
-                else xv = __bfloat162float(reinterpret_cast<const __nv_bfloat16 *>(x)[(size_t)(t0 + tl) * d + c]);
+                float xv[CPT];
+                if constexpr (sizeof(T) == 4) {
+                    xv[0] = reinterpret_cast<const float *>(x)[(size_t)(t0 + tl) * d + c];
+                } else {
+                    const uint32_t w = *reinterpret_cast<const uint32_t *>(
+                        reinterpret_cast<const __nv_bfloat16 *>(x) + (size_t)(t0 + tl) * d + c);
+                    xv[0] = __uint_as_float(w << 16);
+                    xv[CPT - 1] = __uint_as_float(w & 0xFFFF0000u);
+                }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) acc[i] = fmaf(dzs[tl][i], xv, acc[i]);
+                for (int i = 0; i < 8; ++i)
+#pragma unroll
+                    for (int u = 0; u < CPT; ++u) acc[i][u] = fmaf(dzs[tl][i], xv[u], acc[i][u]);
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-                if (g0 + i < N) dwr_partial[((size_t)blockIdx.x * N + g0 + i) * d + c] = acc[i];
+                if (g0 + i < N)
+#pragma unroll
+                    for (int u = 0; u < CPT; ++u)
+                        dwr_partial[((size_t)blockIdx.x * N + g0 + i) * d + c + u] = acc[i][u];
         }
     }
 }
@@ -644,14 +669,15 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
                           const WsPtrs &p, cudaStream_t s, int *launches)
 {
     const int nblk = (T + kRouterTokB - 1) / kRouterTokB;
-    if (dt == MODSE_BF16 && m.N <= 16 && m.d % 64 == 0 && m.k * m.N * 4 <= 128) {
+    if (dt == MODSE_BF16 && m.N <= 16 && m.d % (32 * kRouterKSplit) == 0 && m.k * m.N * 4 <= 128) {
         const int nt = (m.N + 7) / 8;
-        const size_t smem = 128 + (size_t)4 * 32 * nt * 4 * sizeof(float) + (size_t)nt * 8 * (m.d + 8) * 2;
+        const size_t smem = 128 + (size_t)(kRouterKSplit - 1) * 4 * 32 * nt * 4 * sizeof(float) +
+                            (size_t)nt * 8 * (m.d + 8) * 2;
         if (smem <= 200 * 1024) {
             auto kern = nt == 1 ? router_mma_kernel<1> : router_mma_kernel<2>;
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
-            kern<<<nblk, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
+            kern<<<nblk, kRouterMmaThreads, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
                                          p.topk_idx, p.topk_gate, p.block_counts);
             MODSE_LAUNCH_CHECK();
             return cudaSuccess;
@@ -755,7 +781,7 @@ cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *
             (const __nv_bfloat16 *)w_router, dxp, T, m.d, m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz,
             (__nv_bfloat16 *)dx);
     MODSE_LAUNCH_CHECK();
-    dim3 grid(nblk_bwd, (m.d + 255) / 256);
+    dim3 grid(nblk_bwd, dt == MODSE_F32 ? (m.d + 255) / 256 : (m.d + 511) / 512);
     if (dt == MODSE_F32)
         router_dwr_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.topk_idx, p.dz,
                                                       p.dwr_partial);

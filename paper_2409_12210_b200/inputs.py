@@ -46,6 +46,7 @@ CONFIGS = {
     "fwd_8k": LayerConfig("fwd_8k", "bf16", 2048, WIDTHS_700M, 2, 8192, weight_std=0.02, backward=False),
     "train_16k": LayerConfig("train_16k", "bf16", 2048, WIDTHS_700M, 2, 16384, weight_std=0.02),
     "train_16k_equal": LayerConfig("train_16k_equal", "bf16", 2048, WIDTHS_EQUAL, 2, 16384, weight_std=0.02),
+    "train_64k": LayerConfig("train_64k", "bf16", 2048, WIDTHS_700M, 2, 65536, weight_std=0.02),
 }
 
 
