@@ -87,7 +87,9 @@ class LayerInputs:
         return rows
 
 
-def generate(cfg: LayerConfig) -> LayerInputs:
+def generate(cfg: LayerConfig, routing_only: bool = False) -> LayerInputs:
+    """Seeded inputs of `cfg`.  With routing_only the expert weights and dY are left out (empty
+    lists / None); x and W_router are the first two draws, so they are the same either way."""
     rng = np.random.default_rng(cfg.seed)
     d, N, T = cfg.d_model, cfg.n_experts, cfg.n_tokens
 
@@ -99,6 +101,11 @@ def generate(cfg: LayerConfig) -> LayerInputs:
 
     x = normal((T, d), 1.0)
     w_router = normal((N, d), wstd(d))
+    if routing_only:
+        if cfg.router_bias is not None:
+            x[:, -1] = 1.0
+            w_router[:, -1] = np.asarray(cfg.router_bias, dtype=np.float32)
+        return LayerInputs(cfg, to_storage(x, cfg.dtype), to_storage(w_router, cfg.dtype), [], [], [], None, rng)
     w_gate = [normal((h, d), wstd(d)) for h in cfg.ffn_sizes]
     w_up = [normal((h, d), wstd(d)) for h in cfg.ffn_sizes]
     w_down = [normal((d, h), wstd(h)) for h in cfg.ffn_sizes]
