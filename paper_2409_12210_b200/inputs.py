@@ -41,12 +41,22 @@ WIDTHS_RATIO4 = (2240, 9024, 3072, 8192, 3968, 7296, 4800, 6464)
 WIDTHS_TABLE2_700M = (9216, 1024, 8192, 2048, 6144, 4096, 5120, 5120)   # Table 2, 700M x 8
 WIDTHS_TABLE2_300M = (6912, 768, 6144, 1536, 4608, 3072, 3840, 3840)    # Table 2, 300M x 8 (width 1536)
 
+# Router logit offsets of the skewed-routing stress case: assignment shares ~ rank^-1.2 with rank 1 =
+# the widest expert (0.43 of all assignments go to the 8448-wide expert).  Fitted on the seeded train_16k
+# tokens with the reference router by tests/golden/fit_router_bias.py; tests/golden/router_bias_zipf.txt
+# holds the same numbers with the shares reached.
+ZIPF_ROUTER_BIAS = (-2.203125, 0.0, -2.0625, -1.171875, -2.0, -1.53125, -1.8671875, -1.765625)
+
 CONFIGS = {
     "tiny_f32": LayerConfig("tiny_f32", "f32", 64, (96, 160, 112, 144), 2, 256),
     "fwd_8k": LayerConfig("fwd_8k", "bf16", 2048, WIDTHS_700M, 2, 8192, weight_std=0.02, backward=False),
     "train_16k": LayerConfig("train_16k", "bf16", 2048, WIDTHS_700M, 2, 16384, weight_std=0.02),
     "train_16k_equal": LayerConfig("train_16k_equal", "bf16", 2048, WIDTHS_EQUAL, 2, 16384, weight_std=0.02),
     "train_64k": LayerConfig("train_64k", "bf16", 2048, WIDTHS_700M, 2, 65536, weight_std=0.02),
+    "train_16k_skew": LayerConfig("train_16k_skew", "bf16", 2048, WIDTHS_700M, 2, 16384, weight_std=0.02,
+                                  router_bias=ZIPF_ROUTER_BIAS),
+    "train_16k_equal_skew": LayerConfig("train_16k_equal_skew", "bf16", 2048, WIDTHS_EQUAL, 2, 16384,
+                                        weight_std=0.02, router_bias=ZIPF_ROUTER_BIAS),
 }
 
 

@@ -3,6 +3,8 @@
 bench.py times.  The routing tables are compared in full (bit-exact); floating outputs are
 compared on sampled tokens / sampled weight-gradient rows that the fp64 oracle computes one
 by one, and dW_router through the identity dW_router = dz^T x."""
+import os
+
 import numpy as np
 import pytest
 
@@ -59,7 +61,7 @@ def compare(gpu, ora, cfg, backward, discount):
     return errs
 
 
-@pytest.mark.parametrize("name", ["fwd_8k", "train_16k"])
+@pytest.mark.parametrize("name", ["fwd_8k", "train_16k", "train_16k_skew"])
 def test_full_size_sampled_parity(name):
     cfg = I.CONFIGS[name]
     inp, n_redrawn = H.screened(cfg)
@@ -68,7 +70,13 @@ def test_full_size_sampled_parity(name):
     rt = ora["rt"]
     # near-uniform routing, as in the paper's summed-slot shares (every expert 0.118-0.133 of the assignments)
     share = rt.counts / rt.counts.sum()
-    assert share.min() > 0.08 and share.max() < 0.17
+    if cfg.router_bias is None:
+        assert share.min() > 0.08 and share.max() < 0.17
+    else:
+        # stress case: shares ~ rank^-1.2 with the widest expert first (fitted offsets, 1 % of target)
+        want = np.loadtxt(os.path.join(os.path.dirname(__file__), "golden", "router_bias_zipf.txt"), comments=None,
+                          skiprows=2, max_rows=1, usecols=range(3, 11))
+        assert np.max(np.abs(share / want - 1.0)) < 0.02
 
     gpu32 = H.run_gpu(inp, cfg.backward, out_f32=True)
     assert gpu32["status"] == 0
