@@ -215,6 +215,24 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, tq = lane & 3;
     const int grp = warp & 3, kpart = warp >> 2;        // 16-token group; which part of the k range
+    const int t0 = blockIdx.x * kRouterTokB + grp * 16;
+    const int r0 = t0 + g, r1 = t0 + g + 8;
+    const bool v0 = r0 < Ttok, v1 = r1 < Ttok;
+    const uint4 *x0 = reinterpret_cast<const uint4 *>(x + (size_t)(v0 ? r0 : 0) * d + tq * 8);
+    const uint4 *x1 = reinterpret_cast<const uint4 *>(x + (size_t)(v1 ? r1 : 0) * d + tq * 8);
+    const int cbeg = kpart * (d / kRouterKSplit);
+    const int niter = (d / kRouterKSplit) / 32;
+    // The token rows are fetched in batches of UB k-chunks, one batch ahead of the MMAs; the first
+    // batch is in flight while the router matrix is staged in shared memory.
+    constexpr int UB = 4;
+    uint4 xa[UB], xb[UB];
+    const uint4 za = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int u = 0; u < UB; ++u) {
+        const int c0 = cbeg + u * 32;
+        xa[u] = (v0 && u < niter) ? x0[c0 >> 3] : za;
+        xb[u] = (v1 && u < niter) ? x1[c0 >> 3] : za;
+    }
     for (int i = tid; i < k * N; i += kRouterMmaThreads) cnt[i] = 0;
     for (int i = tid * 8; i < NT * 8 * d; i += kRouterMmaThreads * 8) {
         const int r = i / d, c = i % d;
@@ -224,25 +242,31 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
     }
     __syncthreads();
 
-    const int t0 = blockIdx.x * kRouterTokB + grp * 16;
-    const int r0 = t0 + g, r1 = t0 + g + 8;
-    const bool v0 = r0 < Ttok, v1 = r1 < Ttok;
-    const uint4 *x0 = reinterpret_cast<const uint4 *>(x + (size_t)(v0 ? r0 : 0) * d + tq * 8);
-    const uint4 *x1 = reinterpret_cast<const uint4 *>(x + (size_t)(v1 ? r1 : 0) * d + tq * 8);
     float acc[NT][4];
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-    const int cbeg = kpart * (d / kRouterKSplit), cend = cbeg + d / kRouterKSplit;
-#pragma unroll 8
-    for (int c0 = cbeg; c0 < cend; c0 += 32) {
-        const uint4 za = make_uint4(0u, 0u, 0u, 0u);
-        const uint4 xa = v0 ? x0[c0 >> 3] : za;
-        const uint4 xb = v1 ? x1[c0 >> 3] : za;
+    for (int it0 = 0; it0 < niter; it0 += UB) {
+        uint4 ca[UB], cb[UB];
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) {
-            const uint4 w = *reinterpret_cast<const uint4 *>(wsm + (size_t)(nt * 8 + g) * ldw + c0 + tq * 8);
-            mma_bf16_16816(acc[nt], xa.x, xb.x, xa.y, xb.y, w.x, w.y);
-            mma_bf16_16816(acc[nt], xa.z, xb.z, xa.w, xb.w, w.z, w.w);
+        for (int u = 0; u < UB; ++u) { ca[u] = xa[u]; cb[u] = xb[u]; }
+#pragma unroll
+        for (int u = 0; u < UB; ++u) {
+            const int it = it0 + UB + u;
+            const int c0 = cbeg + it * 32;
+            xa[u] = (v0 && it < niter) ? x0[c0 >> 3] : za;
+            xb[u] = (v1 && it < niter) ? x1[c0 >> 3] : za;
+        }
+#pragma unroll
+        for (int u = 0; u < UB; ++u) {
+            const int c0 = cbeg + (it0 + u) * 32;
+            if (it0 + u < niter) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint4 w = *reinterpret_cast<const uint4 *>(wsm + (size_t)(nt * 8 + g) * ldw + c0 + tq * 8);
+                    mma_bf16_16816(acc[nt], ca[u].x, cb[u].x, ca[u].y, cb[u].y, w.x, w.y);
+                    mma_bf16_16816(acc[nt], ca[u].z, cb[u].z, ca[u].w, cb[u].w, w.z, w.w);
+                }
+            }
         }
     }
     // the other warps hand their partial logits to the first warp of the same token group,

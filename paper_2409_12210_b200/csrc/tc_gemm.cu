@@ -338,6 +338,21 @@ __device__ __forceinline__ void store_f32x32(float *dst, const float (&v)[32])
     for (int q = 0; q < 8; ++q) p[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
 }
 
+// Called before the accumulator of a tile is ready: asks L2 for what the epilogue will read from
+// global memory (only the down dgrad reads: the two saved SwiGLU factors of its row).
+template <int KIND>
+__device__ __forceinline__ void epilogue_prefetch(const TcParams &prm, const Tile &t, int row, int c_begin, int c_end)
+{
+    if constexpr (KIND == TcDownDgrad) {
+        for (int c = c_begin; c < c_end; c += 64) {      // one 128-byte line per array covers two 32-column chunks
+            const int col = t.n0 + c;
+            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6);
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.sp + idx));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.sq + idx));
+        }
+    }
+}
+
 // Epilogue of one tile for one thread: accumulator row `row`, columns [c_begin, c_end).
 template <int KIND>
 __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t, uint32_t tacc, int row, int c_begin,
@@ -621,10 +636,11 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
             const Tile t = decode_tile<KIND>(prm, st, tile, cursor);
             const int acc = it & 1;
             const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            const int chalf = t.ncols >> 1;            // a multiple of 32: ncols is a multiple of 64
+            epilogue_prefetch<KIND>(prm, t, row, half * chalf, (half + 1) * chalf);
             if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, prm.status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
-            const int chalf = t.ncols >> 1;            // a multiple of 32: ncols is a multiple of 64
             epilogue_row<KIND>(prm, t, tacc, row, half * chalf, (half + 1) * chalf);
             tc_fence_before();
             mbar_arrive(smem_u32(&st->tmem_empty[acc]));
