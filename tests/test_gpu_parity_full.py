@@ -17,7 +17,7 @@ pytestmark = pytest.mark.gpu
 
 TOL_BF16 = 2e-2
 N_TOKENS_SAMPLED = 48
-N_ROWS_SAMPLED = 24
+ROWS_PER_EXPERT = 4
 
 
 def f64(a):
@@ -36,7 +36,7 @@ def oracle_samples(inp, backward, seed=7):
         dy = f64(inp.dy)
         out["dx"], out["dg"], dz = O.backward_tokens(x, wr, pw, rt, dy, sel)
         out["dz"] = np.take_along_axis(dz, rt.topk_idx[sel].astype(np.int64), 1)
-        rows_e = rng.integers(0, cfg.n_experts, N_ROWS_SAMPLED).astype(np.int32)
+        rows_e = np.repeat(np.arange(cfg.n_experts), ROWS_PER_EXPERT).astype(np.int32)
         rows_r = np.array([rng.integers(0, cfg.ffn_sizes[e]) for e in rows_e], np.int32)
         out["rows_e"], out["rows_r"] = rows_e, rows_r
         out["dwg"], out["dwu"], out["dwd"] = O.wgrad_rows(x, pw, rt, dy, rows_e, rows_r)
@@ -50,12 +50,24 @@ def compare(gpu, ora, cfg, backward, discount):
     if backward:
         hoff = np.concatenate([[0], np.cumsum(cfg.ffn_sizes)])
         rows = hoff[ora["rows_e"]] + ora["rows_r"]
-        errs["dx"] = err(gpu["dx"][sel], ora["dx"])
+        nd = cfg.d_model if cfg.router_bias is None else cfg.d_model - 1
+        errs["dx"] = err(gpu["dx"][sel][:, :nd], ora["dx"][:, :nd])
+        if cfg.router_bias is not None:
+            # The stress case feeds the logit offsets through a constant input channel whose router
+            # weights are ~100x the others, so dx of that one channel is sum_j dz_j b_j: it carries
+            # the relative error of dz (bf16-level, bounded above by its own entry) times |b|, and
+            # is measured against its own RMS.
+            errs["dx_bias_channel"] = err(gpu["dx"][sel][:, nd:], ora["dx"][:, nd:])
         errs["dg"] = H.rel_err(gpu["dg"][sel], ora["dg"])
         errs["dz"] = H.rel_err(gpu["dz"][sel], ora["dz"])
-        errs["dw_gate"] = err(gpu["dw_gate"][rows], ora["dwg"])
-        errs["dw_up"] = err(gpu["dw_up"][rows], ora["dwu"])
-        errs["dw_down"] = err(gpu["dw_down"][:, rows].T, ora["dwd"])
+        # each expert's weight gradient is a tensor of its own (their magnitudes differ with the token
+        # counts): the sampled rows are normalised expert by expert and the worst expert is reported
+        per_expert = lambda got, ref: max(err(got[ora["rows_e"] == e], ref[ora["rows_e"] == e])
+                                          for e in range(cfg.n_experts))
+        errs["dw_gate"] = per_expert(gpu["dw_gate"][rows], ora["dwg"])
+        errs["dw_up"] = per_expert(gpu["dw_up"][rows], ora["dwu"])
+        errs["dw_down"] = per_expert(gpu["dw_down"][:, rows].T, ora["dwd"])
+    print(f"{cfg.name} {'bf16' if discount else 'fp32'} outputs:", {k: round(v, 4) for k, v in errs.items()})
     bad = {k: v for k, v in errs.items() if not (v <= TOL_BF16)}
     assert not bad, f"over tolerance {TOL_BF16}: {bad} (all: {errs})"
     return errs
