@@ -70,6 +70,8 @@ constexpr int kThreads = 320;                   // TMA warp, MMA warp, eight epi
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
+constexpr int kEpiRowBytes = 64 + 16;            // a 32-element bf16 chunk of one row, skewed by 16 bytes
+constexpr int kEpiWarpBytes = 32 * kEpiRowBytes;
 
 struct TcParams {
     LayerMeta meta;
@@ -87,6 +89,7 @@ struct TcParams {
 
 // dynamic shared memory map (after 1024-byte alignment)
 struct SmemTail {
+    unsigned char epi_stage[8][kEpiWarpBytes];   // one transposing buffer per epilogue warp
     unsigned long long full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
     unsigned int tmem_base;
     int abort_flag;
@@ -331,6 +334,64 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16 *dst, const float (&
     }
 }
 
+// A warp's 32 threads each hold 32 bf16 values of their own row (64 bytes); the rows are
+// `row_stride` elements apart in global memory.  Storing (or loading) them row by row would touch
+// 32 lines with 16 bytes each per instruction, so the chunk is transposed through shared memory:
+// afterwards four neighbouring lanes cover the 64 bytes of one row and an instruction moves eight
+// whole 64-byte row segments.  `own` points at this thread's own row chunk.
+__device__ __forceinline__ void store_bf16x32_staged(unsigned char *stg, int lane, __nv_bfloat16 *own, long long row_stride,
+                                                     const float (&v)[32])
+{
+    uint4 *mine = reinterpret_cast<uint4 *>(stg + lane * kEpiRowBytes);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t *>(&t);
+        }
+        mine[q] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __syncwarp();
+    const int q = lane & 3;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int rr = 8 * j + (lane >> 2);
+        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * kEpiRowBytes + q * 16);
+        *reinterpret_cast<uint4 *>(own + (long long)(rr - lane) * row_stride + q * 8) = val;
+    }
+    __syncwarp();
+}
+
+// Transposed (coalesced) load of a warp's 32 row chunks; raw[j] belongs to row 8j + lane/4.
+__device__ __forceinline__ void load_bf16x32_transposed(const __nv_bfloat16 *own, long long row_stride, int lane,
+                                                        uint4 (&raw)[4])
+{
+    const int q = lane & 3;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int rr = 8 * j + (lane >> 2);
+        raw[j] = *reinterpret_cast<const uint4 *>(own + (long long)(rr - lane) * row_stride + q * 8);
+    }
+}
+
+// Hands every thread the 64 bytes of its own row out of a transposed load.
+__device__ __forceinline__ void untranspose_rows(unsigned char *stg, int lane, const uint4 (&raw)[4], uint4 (&own)[4])
+{
+    const int q = lane & 3;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int rr = 8 * j + (lane >> 2);
+        *reinterpret_cast<uint4 *>(stg + rr * kEpiRowBytes + q * 16) = raw[j];
+    }
+    __syncwarp();
+    const uint4 *mine = reinterpret_cast<const uint4 *>(stg + lane * kEpiRowBytes);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) own[i] = mine[i];
+    __syncwarp();
+}
+
 __device__ __forceinline__ void store_f32x32(float *dst, const float (&v)[32])
 {
     float4 *p = reinterpret_cast<float4 *>(dst);
@@ -356,8 +417,9 @@ __device__ __forceinline__ void epilogue_prefetch(const TcParams &prm, const Til
 // Epilogue of one tile for one thread: accumulator row `row`, columns [c_begin, c_end).
 template <int KIND>
 __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t, uint32_t tacc, int row, int c_begin,
-                                             int c_end)
+                                             int c_end, unsigned char *stg)
 {
+    const int lane = row & 31;
     const int d = prm.meta.d, S = prm.meta.S;
     const bool have_acc = t.nk > 0;
     auto panel_index = [&](int c) {
@@ -383,8 +445,8 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
                     sp[i] = bv * sg * (1.0f + av * (1.0f - sg));
                     hm[i] = gate * (sq[i] * bv);
                 }
-                store_bf16x32(prm.sp + idx, sp);
-                store_bf16x32(prm.sq + idx, sq);
+                store_bf16x32_staged(stg, lane, prm.sp + idx, 64, sp);
+                store_bf16x32_staged(stg, lane, prm.sq + idx, 64, sq);
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
@@ -392,7 +454,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
                     hm[i] = gate * (av * (1.0f / (1.0f + __expf(-av))) * bv);
                 }
             }
-            store_bf16x32(prm.hm + idx, hm);
+            store_bf16x32_staged(stg, lane, prm.hm + idx, 64, hm);
         }
     } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
         float *out = (KIND == TcDown ? prm.o : prm.dxp) + (size_t)(t.prow0 + t.m0 + row) * d + t.n0;
@@ -409,13 +471,11 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
         // dA = dHm * sp, dB = dHm * sq with dHm = gate * acc; the saved factors of the next
         // chunk are fetched while this one is computed
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
-        uint4 praw[4], qraw[4];
+        uint4 praw[4], qraw[4];            // transposed: entry j belongs to row 8j + lane/4 of this warp
         {
             const size_t idx = panel_index(c_begin);
-            const uint4 *pp = reinterpret_cast<const uint4 *>(prm.sp + idx);
-            const uint4 *qq = reinterpret_cast<const uint4 *>(prm.sq + idx);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { praw[i] = pp[i]; qraw[i] = qq[i]; }
+            load_bf16x32_transposed(prm.sp + idx, 64, lane, praw);
+            load_bf16x32_transposed(prm.sq + idx, 64, lane, qraw);
         }
         for (int c = c_begin; c < c_end; c += 32) {
             uint32_t r[32];
@@ -424,18 +484,19 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             const bool more = c + 32 < c_end;
             if (more) {
                 const size_t nidx = panel_index(c + 32);
-                const uint4 *pp = reinterpret_cast<const uint4 *>(prm.sp + nidx);
-                const uint4 *qq = reinterpret_cast<const uint4 *>(prm.sq + nidx);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { pn[i] = pp[i]; qn[i] = qq[i]; }
+                load_bf16x32_transposed(prm.sp + nidx, 64, lane, pn);
+                load_bf16x32_transposed(prm.sq + nidx, 64, lane, qn);
             }
+            uint4 pown[4], qown[4];
+            untranspose_rows(stg, lane, praw, pown);
+            untranspose_rows(stg, lane, qraw, qown);
             tmem_ld_wait();
             const size_t idx = panel_index(c);
             float da[32], db[32];
 #pragma unroll
             for (int q4 = 0; q4 < 4; ++q4) {
-                const uint32_t pw[4] = {praw[q4].x, praw[q4].y, praw[q4].z, praw[q4].w};
-                const uint32_t qw[4] = {qraw[q4].x, qraw[q4].y, qraw[q4].z, qraw[q4].w};
+                const uint32_t pw[4] = {pown[q4].x, pown[q4].y, pown[q4].z, pown[q4].w};
+                const uint32_t qw[4] = {qown[q4].x, qown[q4].y, qown[q4].z, qown[q4].w};
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int e0 = q4 * 8 + 2 * i;
@@ -446,8 +507,8 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
                     db[e0 + 1] = dh1 * __uint_as_float(qw[i] & 0xFFFF0000u);
                 }
             }
-            store_bf16x32(prm.da + idx, da);
-            store_bf16x32(prm.db + idx, db);
+            store_bf16x32_staged(stg, lane, prm.da + idx, 64, da);
+            store_bf16x32_staged(stg, lane, prm.db + idx, 64, db);
             if (more) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) { praw[i] = pn[i]; qraw[i] = qn[i]; }
@@ -641,7 +702,7 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
             if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, prm.status)) { ok = false; break; }
             tc_fence_after();
             const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
-            epilogue_row<KIND>(prm, t, tacc, row, half * chalf, (half + 1) * chalf);
+            epilogue_row<KIND>(prm, t, tacc, row, half * chalf, (half + 1) * chalf, st->epi_stage[warp - 2]);
             tc_fence_before();
             mbar_arrive(smem_u32(&st->tmem_empty[acc]));
         }
@@ -675,6 +736,7 @@ constexpr int kARegion2 = 2 * kBoxBytes;
 constexpr int kBRegion2 = 2 * kBoxBytes;
 constexpr int kStageBytes2 = kARegion2 + kBRegion2;   // 32 KB
 struct SmemTail2 {
+    unsigned char epi_stage[8][kEpiWarpBytes];   // one transposing buffer per epilogue warp
     unsigned long long full[kStages2], empty[kStages2], tmem_full[2], tmem_empty[2];
     unsigned int tmem_base;
     int abort_flag;
@@ -988,7 +1050,7 @@ tc_grouped_gemm_pair(const __grid_constant__ TcMaps maps, const __grid_constant_
                 const int span = (KIND == TcUpGate) ? t.ncols : t.n_mma;
                 const int chalf = span >> 1;
                 const int c0 = half * chalf, c1 = min((half + 1) * chalf, t.ncols);
-                if (c0 < c1) epilogue_row<KIND>(prm, t, tacc, row, c0, c1);
+                if (c0 < c1) epilogue_row<KIND>(prm, t, tacc, row, c0, c1, st->epi_stage[warp - 2]);
             }
             tc_fence_before();
             __syncwarp();
@@ -1026,6 +1088,7 @@ constexpr int kStagesW = 3;
 constexpr int kARegionW = 4 * kBoxBytes;            // two halves of 128 rows x 64 K
 constexpr int kStageBytesW = kARegionW + kBRegion;  // 64 KB
 struct SmemTailW {
+    unsigned char epi_stage[8][kEpiWarpBytes];   // one transposing buffer per epilogue warp
     unsigned long long full[kStagesW], empty[kStagesW], tmem_full[1], tmem_empty[2];
     unsigned int tmem_base;
     int abort_flag;
@@ -1308,12 +1371,13 @@ tc_grouped_gemm_wide(const __grid_constant__ TcMaps maps, const __grid_constant_
             tc_fence_after();
             const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16);
             const int chalf = t0.ncols >> 1;
-            epilogue_row<KIND>(prm, t0, tacc, row, half * chalf, (half + 1) * chalf);
+            epilogue_row<KIND>(prm, t0, tacc, row, half * chalf, (half + 1) * chalf, st->epi_stage[warp - 2]);
             tc_fence_before();
             mbar_arrive(smem_u32(&st->tmem_empty[0]));
             if (t0.a_boxes_peer > 0) {
                 const Tile t1 = second_half(t0);
-                epilogue_row<KIND>(prm, t1, tacc + kAccCols, row, half * chalf, (half + 1) * chalf);
+                epilogue_row<KIND>(prm, t1, tacc + kAccCols, row, half * chalf, (half + 1) * chalf,
+                                   st->epi_stage[warp - 2]);
                 tc_fence_before();
                 mbar_arrive(smem_u32(&st->tmem_empty[1]));
             }
