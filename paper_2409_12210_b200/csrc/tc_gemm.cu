@@ -319,49 +319,59 @@ __device__ __forceinline__ void issue_loads(const TcMaps &maps, const Tile &t, i
     }
 }
 
-__device__ __forceinline__ void store_bf16x32(__nv_bfloat16 *dst, const float (&v)[32])
-{
-    uint4 *p = reinterpret_cast<uint4 *>(dst);
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 t = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
-            w[i] = *reinterpret_cast<uint32_t *>(&t);
-        }
-        p[q] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-}
-
 // A warp's 32 threads each hold 32 bf16 values of their own row (64 bytes); the rows are
 // `row_stride` elements apart in global memory.  Storing (or loading) them row by row would touch
 // 32 lines with 16 bytes each per instruction, so the chunk is transposed through shared memory:
 // afterwards four neighbouring lanes cover the 64 bytes of one row and an instruction moves eight
 // whole 64-byte row segments.  `own` points at this thread's own row chunk.
-__device__ __forceinline__ void store_bf16x32_staged(unsigned char *stg, int lane, __nv_bfloat16 *own, long long row_stride,
-                                                     const float (&v)[32])
+// rows_valid: rows of this warp (0..32, counted from the warp's first row) that may be written.
+__device__ __forceinline__ void store_u4x4_staged(unsigned char *stg, int lane, unsigned char *own, long long row_stride_bytes,
+                                                  const uint4 (&w)[4], int rows_valid)
 {
     uint4 *mine = reinterpret_cast<uint4 *>(stg + lane * kEpiRowBytes);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 t = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
-            w[i] = *reinterpret_cast<uint32_t *>(&t);
-        }
-        mine[q] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
+    for (int q = 0; q < 4; ++q) mine[q] = w[q];
     __syncwarp();
     const int q = lane & 3;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int rr = 8 * j + (lane >> 2);
         const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * kEpiRowBytes + q * 16);
-        *reinterpret_cast<uint4 *>(own + (long long)(rr - lane) * row_stride + q * 8) = val;
+        if (rr < rows_valid) *reinterpret_cast<uint4 *>(own + (long long)(rr - lane) * row_stride_bytes + q * 16) = val;
     }
     __syncwarp();
+}
+
+__device__ __forceinline__ void store_bf16x32_staged(unsigned char *stg, int lane, __nv_bfloat16 *own, long long row_stride,
+                                                     const float (&v)[32], int rows_valid = 32)
+{
+    uint4 w4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t *>(&t);
+        }
+        w4[q] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    store_u4x4_staged(stg, lane, reinterpret_cast<unsigned char *>(own), row_stride * 2, w4, rows_valid);
+}
+
+// 32 fp32 values per row (128 bytes) go out as two 64-byte halves.
+__device__ __forceinline__ void store_f32x32_staged(unsigned char *stg, int lane, float *own, long long row_stride,
+                                                    const float (&v)[32], int rows_valid = 32)
+{
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        uint4 w4[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            w4[q] = make_uint4(__float_as_uint(v[hh * 16 + 4 * q]), __float_as_uint(v[hh * 16 + 4 * q + 1]),
+                               __float_as_uint(v[hh * 16 + 4 * q + 2]), __float_as_uint(v[hh * 16 + 4 * q + 3]));
+        store_u4x4_staged(stg, lane, reinterpret_cast<unsigned char *>(own + hh * 16), row_stride * 4, w4, rows_valid);
+    }
 }
 
 // Transposed (coalesced) load of a warp's 32 row chunks; raw[j] belongs to row 8j + lane/4.
@@ -390,13 +400,6 @@ __device__ __forceinline__ void untranspose_rows(unsigned char *stg, int lane, c
 #pragma unroll
     for (int i = 0; i < 4; ++i) own[i] = mine[i];
     __syncwarp();
-}
-
-__device__ __forceinline__ void store_f32x32(float *dst, const float (&v)[32])
-{
-    float4 *p = reinterpret_cast<float4 *>(dst);
-#pragma unroll
-    for (int q = 0; q < 8; ++q) p[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
 }
 
 // Called before the accumulator of a tile is ready: asks L2 for what the epilogue will read from
@@ -465,7 +468,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-            store_f32x32(out + c, v);
+            store_f32x32_staged(stg, lane, out + c, d, v);
         }
     } else if constexpr (KIND == TcDownDgrad) {
         // dA = dHm * sp, dB = dHm * sq with dHm = gate * acc; the saved factors of the next
@@ -528,8 +531,8 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
             }
-            if (prm.out_f32) store_f32x32(reinterpret_cast<float *>(prm.dw_down) + oidx + c, v);
-            else store_bf16x32(prm.dw_down + oidx + c, v);
+            if (prm.out_f32) store_f32x32_staged(stg, lane, reinterpret_cast<float *>(prm.dw_down) + oidx + c, S, v);
+            else store_bf16x32_staged(stg, lane, prm.dw_down + oidx + c, S, v);
         }
     } else {
         __nv_bfloat16 *obase = t.which ? prm.dw_up : prm.dw_gate;
@@ -546,10 +549,9 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
             }
-            if (row < t.mrows) {
-                if (prm.out_f32) store_f32x32(reinterpret_cast<float *>(obase) + oidx + c, v);
-                else store_bf16x32(obase + oidx + c, v);
-            }
+            const int rows_valid = t.mrows - (row - lane);      // rows of this warp inside the expert's width
+            if (prm.out_f32) store_f32x32_staged(stg, lane, reinterpret_cast<float *>(obase) + oidx + c, d, v, rows_valid);
+            else store_bf16x32_staged(stg, lane, obase + oidx + c, d, v, rows_valid);
         }
     }
 }
