@@ -151,6 +151,25 @@ modse_status_t modse_check_device_status(modse_layer_t *layer, const void *works
  * enqueued (for launch accounting in benchmarks).                            */
 int modse_last_launch_count(const modse_layer_t *layer);
 
+/* Auxiliary load-balance loss of Sec. 3.2, Eq. 7-10 (the Switch-Transformer loss):
+ *   L_a = alpha * N * sum_i f_i * P_i,
+ * p(x) = softmax over all N router logits, f_i = fraction of tokens whose largest
+ * probability is expert i (Eq. 8; equals the slot-0 count / T), P_i = mean of p_i
+ * over the batch (Eq. 10).
+ *
+ * modse_aux_loss evaluates it for the batch of the last modse_forward on this layer
+ * and workspace: loss (1 float), f [N] and P [N] are device pointers written on the
+ * stream (f and P may be NULL).
+ *
+ * modse_set_aux_loss(alpha) makes the following modse_backward calls differentiate
+ * the objective  sum(dy * y) + L_a : dx and dw_router receive, in addition,
+ * dL_a/dz[t,m] = (alpha N / T) p_m (f_m - sum_i f_i p_i) for every expert m (f is
+ * piecewise constant and is held fixed).  alpha = 0 (default) switches it off.
+ * The fp32 dz returned by modse_get_gate_grads stays the layer-output part only. */
+modse_status_t modse_aux_loss(modse_layer_t *layer, const void *workspace, int n_tokens, float alpha, float *loss,
+                              float *f, float *P, void *cuda_stream);
+modse_status_t modse_set_aux_loss(modse_layer_t *layer, float alpha);
+
 /* Output precision of a bf16 layer.  Off (default): y, dx and the expert weight
  * gradients are bf16 like the inputs.  On: the same fp32 accumulators are
  * written as fp32 instead ([T,d] y and dx, [S,d]/[d,S] weight gradients of 4

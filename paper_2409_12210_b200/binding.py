@@ -87,6 +87,10 @@ def load():
     lib.modse_route_static_scratch.restype = ci
     lib.modse_route_static_scratch.argtypes = [ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.modse_route_static_scratch_capacity.restype = sz
+    lib.modse_aux_loss.restype = ci
+    lib.modse_aux_loss.argtypes = [vp, vp, ci, ctypes.c_float, vp, vp, vp, vp]
+    lib.modse_set_aux_loss.restype = ci
+    lib.modse_set_aux_loss.argtypes = [vp, ctypes.c_float]
     lib.modse_set_output_f32.restype = ci
     lib.modse_set_output_f32.argtypes = [vp, ci]
     lib.modse_stage_timing_begin.restype = ci
@@ -255,6 +259,24 @@ class ModseLayer:
 
     def check_device_status(self, workspace) -> int:
         return int(load().modse_check_device_status(self._h, workspace.data_ptr(), self._stream()))
+
+    def set_aux_loss(self, alpha: float) -> None:
+        st = load().modse_set_aux_loss(self._h, float(alpha))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_set_aux_loss")
+
+    def aux_loss(self, workspace, n_tokens: int, alpha: float):
+        """(loss [1], f [N], P [N]) device tensors of the auxiliary load-balance loss (Eq. 7-10)."""
+        import torch
+        dev = workspace.device
+        loss = torch.empty(1, dtype=torch.float32, device=dev)
+        f = torch.empty(self.n_experts, dtype=torch.float32, device=dev)
+        P = torch.empty(self.n_experts, dtype=torch.float32, device=dev)
+        st = load().modse_aux_loss(self._h, workspace.data_ptr(), n_tokens, float(alpha), loss.data_ptr(),
+                                   f.data_ptr(), P.data_ptr(), self._stream())
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_aux_loss")
+        return loss, f, P
 
     def set_output_f32(self, on: bool) -> None:
         st = load().modse_set_output_f32(self._h, int(bool(on)))

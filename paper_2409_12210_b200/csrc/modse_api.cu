@@ -17,6 +17,7 @@ struct modse_layer {
     int fwd_dtype = -1;
     int fwd_saved = 0;
     int last_launches = 0;
+    float aux_alpha = 0.f;        // coefficient of the auxiliary load-balance loss added to the objective in backward
     int out_f32 = 0;              // bf16 layers: write y, dx and expert weight gradients as fp32
     modse::TcPlan tc;             // device facts of the bf16 path
     // optional per-stage device timing: events [call][stage][start/stop]
@@ -58,6 +59,8 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
     L.ptoken_of = take((size_t)L.Pmax * 4);
     L.pgate = take((size_t)L.Pmax * 4);
     L.block_counts = take((size_t)L.nblk * m.k * N * 4);
+    L.logits = take((size_t)T * N * 4);
+    L.aux_partial = take((size_t)L.nblk_bwd * N * 4);
     L.xp = take((size_t)L.Pmax * m.d * esz);
     L.hm = take(L.hb * esz);
     L.o = take((size_t)L.Pmax * m.d * 4);     // fp32 for every layer type
@@ -98,6 +101,8 @@ WsPtrs carve(void *ws, const WsLayout &L)
     p.ptoken_of = (int *)(b + L.ptoken_of);
     p.pgate = (float *)(b + L.pgate);
     p.block_counts = (int *)(b + L.block_counts);
+    p.logits = (float *)(b + L.logits);
+    p.aux_partial = (float *)(b + L.aux_partial);
     p.dg = (float *)(b + L.dg);
     p.dz = (float *)(b + L.dz);
     p.dwr_partial = (float *)(b + L.dwr_partial);
@@ -375,7 +380,8 @@ modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const m
         MODSE_STAGE(tm, 10, tc_launch(layer->tc, TcUpGateWgrad, maps, m, p, wgrads, true, of32, s, &launches));
     }
     MODSE_STAGE(tm, 11, launch_router_bwd(dtype, m, x, weights->w_router, n_tokens, L.nblk_bwd, p, dx, of32,
-                                          static_cast<float *>(wgrads->dw_router), s, &launches));
+                                          static_cast<float *>(wgrads->dw_router),
+                                          layer->aux_alpha * (float)m.N / (float)n_tokens, s, &launches));
     layer->last_launches = launches;
     return MODSE_OK;
 }
@@ -427,6 +433,28 @@ modse_status_t modse_check_device_status(modse_layer_t *layer, const void *works
 }
 
 int modse_last_launch_count(const modse_layer_t *layer) { return layer ? layer->last_launches : 0; }
+
+modse_status_t modse_set_aux_loss(modse_layer_t *layer, float alpha)
+{
+    if (layer == nullptr || !(alpha >= 0.f)) return MODSE_ERR_INVALID_ARG;
+    layer->aux_alpha = alpha;
+    return MODSE_OK;
+}
+
+modse_status_t modse_aux_loss(modse_layer_t *layer, const void *workspace, int n_tokens, float alpha, float *loss,
+                              float *f, float *P, void *cuda_stream)
+{
+    if (layer == nullptr || workspace == nullptr || n_tokens < 1 || loss == nullptr) return MODSE_ERR_INVALID_ARG;
+    if (layer->fwd_ws != workspace || layer->fwd_tokens != n_tokens) return MODSE_ERR_STATE;
+    const WsLayout L = make_layout(layer->meta, layer->h_desc.data(), layer->fwd_dtype == MODSE_F32 ? 4 : 2,
+                                   n_tokens, layer->fwd_saved != 0);
+    const WsPtrs p = carve(const_cast<void *>(workspace), L);
+    int launches = 0;
+    MODSE_CUDA(launch_aux_loss(layer->meta, n_tokens, L.nblk_bwd, p, alpha, loss, f, P,
+                               static_cast<cudaStream_t>(cuda_stream), &launches));
+    layer->last_launches = launches;
+    return MODSE_OK;
+}
 
 modse_status_t modse_set_output_f32(modse_layer_t *layer, int on)
 {

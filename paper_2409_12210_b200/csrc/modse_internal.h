@@ -31,7 +31,7 @@ struct WsLayout {
     int T, R, Pmax, nblk, nblk_bwd;
     size_t hb;   // element capacity of each [padded rows x h_e] activation buffer
     size_t status, topk_idx, topk_gate, counts, counts_slot, offsets, poffsets, ebase, row_of, token_of,
-        prow_of, ptoken_of, pgate, block_counts, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
+        prow_of, ptoken_of, pgate, block_counts, logits, aux_partial, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
         total;
 };
 
@@ -44,6 +44,8 @@ struct WsPtrs {
     int *row_of, *token_of, *prow_of, *ptoken_of;
     float *pgate;
     int *block_counts;
+    float *logits;       // [T,N] router logits (may be null: not stored)
+    float *aux_partial;  // [nblk_bwd][N] partial sums of the router probabilities
     float *dg, *dz, *dwr_partial;
     void *xp, *a_pre, *b_pre, *hm, *o, *dyp, *da, *db, *dxp;
 };
@@ -61,9 +63,13 @@ cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const Ws
                            cudaStream_t s, int *launches);
 cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, const WsPtrs &p,
                               cudaStream_t s, int *launches);
+// aux_scale = alpha * N / T of the auxiliary load-balance loss (Eq. 7), 0 when it is not part of the objective
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
                               int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
-                              cudaStream_t s, int *launches);
+                              float aux_scale, cudaStream_t s, int *launches);
+// L_a = alpha N sum_i f_i P_i (Eq. 7-10) from the stored logits and the slot-0 histogram
+cudaError_t launch_aux_loss(const LayerMeta &m, int T, int nblk_bwd, const WsPtrs &p, float alpha, float *loss,
+                            float *f, float *P, cudaStream_t s, int *launches);
 
 // ---- fp32-FMA grouped GEMMs and SwiGLU elementwise (simt_gemm.cu) ----
 enum GemmKind : int {

@@ -95,6 +95,7 @@ extern "C" modse_status_t modse_route_static_scratch(modse_dtype_t dtype, int d_
     p.ptoken_of = reinterpret_cast<int *>(base + L.ptoken_of);
     p.pgate = reinterpret_cast<float *>(base + L.pgate);
     p.block_counts = reinterpret_cast<int *>(base + L.block_counts);
+    p.logits = nullptr;                             // the logits themselves are not kept
     p.topk_idx = topk_idx;
     p.topk_gate = topk_gate;
     p.counts = counts;

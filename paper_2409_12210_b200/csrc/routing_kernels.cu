@@ -76,7 +76,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok, int d, int N, int k,
               int *__restrict__ topk_idx, float *__restrict__ topk_gate, int *__restrict__ block_counts,
-              int w_in_smem)
+              float *__restrict__ logits, int w_in_smem)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int Npad = (N + 3) & ~3;
@@ -125,6 +125,8 @@ router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok,
             }
         }
         __syncwarp();
+        if (logits != nullptr)
+            for (int i = lane; i < N; i += 32) logits[(size_t)t * N + i] = z[i];
         // KeepTopK: k rounds of arg-max over the logits not yet taken; the pair
         // (value, index) is ordered so that equal values prefer the lower index.
         float zsel[2] = {0.f, 0.f};
@@ -204,7 +206,7 @@ template <int NT>
 __global__ void __launch_bounds__(kRouterMmaThreads)
 router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w_router, int Ttok, int d,
                   int N, int k, int *__restrict__ topk_idx, float *__restrict__ topk_gate,
-                  int *__restrict__ block_counts)
+                  int *__restrict__ block_counts, float *__restrict__ logits)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     int *cnt = reinterpret_cast<int *>(smem_raw);                                   // [k*N], padded to 128 bytes
@@ -288,6 +290,15 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
                 for (int u = 0; u < 4; ++u)
                     acc[nt][u] += part[((((q - 1) * 4 + grp) * 32 + lane) * NT + nt) * 4 + u];
         // acc[nt][0..1]: token r0, experts nt*8 + 2tq, +1;  acc[nt][2..3]: token r1, same experts
+        if (logits != nullptr) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int t = (u & 2) ? r1 : r0, e = nt * 8 + 2 * tq + (u & 1);
+                    if (t < Ttok && e < N) logits[(size_t)t * N + e] = acc[nt][u];
+                }
+        }
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
             const int t = half ? r1 : r0;
@@ -558,6 +569,76 @@ dg_permute_kernel(const T *__restrict__ dy, const float *__restrict__ o, int Tto
 }
 
 // ---------------------------------------------------------------------------
+// Auxiliary load-balance loss (Sec. 3.2, Eq. 7-10): L_a = alpha N sum_i f_i P_i with
+// p(x) = softmax over all N logits, f_i = share of tokens whose largest probability is
+// expert i (= slot-0 count / T), P_i = mean of p_i.  aux_partial_kernel sums p_i over
+// blocks of 128 tokens (token order inside a block, block order in aux_final_kernel).
+// Its gradient w.r.t. the logits, with f held constant (f is piecewise constant):
+//   dL_a/dz[t,m] = (alpha N / T) p_m (f_m - sum_i f_i p_i).
+// ---------------------------------------------------------------------------
+// softmax statistics of one token: max logit, 1/sum exp, and sum_i f_i p_i
+__device__ __forceinline__ void token_softmax_stats(const float *__restrict__ z, const int *__restrict__ counts_slot,
+                                                    int N, float inv_T, float &zmax, float &inv_den, float &fp)
+{
+    zmax = z[0];
+    for (int i = 1; i < N; ++i) zmax = fmaxf(zmax, z[i]);
+    float den = 0.f, acc = 0.f;
+    for (int i = 0; i < N; ++i) {
+        const float e = expf(z[i] - zmax);
+        den += e;
+        acc = fmaf((float)counts_slot[i] * inv_T, e, acc);
+    }
+    inv_den = 1.0f / den;
+    fp = acc * inv_den;
+}
+
+__global__ void __launch_bounds__(128)
+aux_partial_kernel(const float *__restrict__ logits, int Ttok, int N, float *__restrict__ partial)
+{
+    __shared__ float red[4];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t = blockIdx.x * kRouterBwdTokB + tid;
+    const bool ok = t < Ttok;
+    const float *z = logits + (size_t)(ok ? t : 0) * N;
+    float zmax = z[0];
+    for (int i = 1; i < N; ++i) zmax = fmaxf(zmax, z[i]);
+    float den = 0.f;
+    for (int i = 0; i < N; ++i) den += expf(z[i] - zmax);
+    const float inv = ok ? 1.0f / den : 0.f;
+    for (int i = 0; i < N; ++i) {
+        float v = expf(z[i] - zmax) * inv;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        if (lane == 0) red[warp] = v;
+        __syncthreads();
+        if (tid == 0) partial[(size_t)blockIdx.x * N + i] = (red[0] + red[1]) + (red[2] + red[3]);
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(256)
+aux_final_kernel(const float *__restrict__ partial, int nblk, const int *__restrict__ counts_slot, int Ttok, int N,
+                 float alpha, float *__restrict__ loss, float *__restrict__ f_out, float *__restrict__ P_out)
+{
+    __shared__ float fP[kMaxExperts];
+    const int i = threadIdx.x;
+    if (i < N) {
+        float s = 0.f;
+        for (int b = 0; b < nblk; ++b) s += partial[(size_t)b * N + i];
+        const float P = s / (float)Ttok, f = (float)counts_slot[i] / (float)Ttok;
+        if (f_out) f_out[i] = f;
+        if (P_out) P_out[i] = P;
+        fP[i] = f * P;
+    }
+    __syncthreads();
+    if (i == 0) {
+        float acc = 0.f;
+        for (int e = 0; e < N; ++e) acc += fP[e];
+        *loss = alpha * (float)N * acc;
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Router backward, part 1 (warp per token): s = sum_j g_j dg_j,
 // dz_j = g_j (dg_j - s), dx_t = sum_j dxp[row_j] + sum_j dz_j W_router[e_j].
 // ---------------------------------------------------------------------------
@@ -566,7 +647,8 @@ __global__ void __launch_bounds__(256)
 router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, int Ttok, int d, int k,
                  const int *__restrict__ topk_idx, const float *__restrict__ topk_gate,
                  const int *__restrict__ prow_of, const float *__restrict__ dg, float *__restrict__ dz,
-                 TO *__restrict__ dx)
+                 TO *__restrict__ dx, int N, const float *__restrict__ logits, const int *__restrict__ counts_slot,
+                 float aux_scale)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * 8 + warp;
@@ -583,6 +665,11 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
     dzv[0] = g[0] * (dgv[0] - s);
     dzv[1] = g[1] * (dgv[1] - s);
     if (lane < k) dz[(size_t)t * k + lane] = dzv[lane];
+    // auxiliary loss: every expert's logit gets a gradient (computed by all lanes alike)
+    float zmax = 0.f, inv_den = 0.f, fp = 0.f;
+    const float *zt = logits + (size_t)t * N;
+    const float inv_T = 1.0f / (float)Ttok;
+    if (aux_scale != 0.f) token_softmax_stats(zt, counts_slot, N, inv_T, zmax, inv_den, fp);
     for (int c = lane * 8; c < d; c += 256) {
         float a[8], out[8], wv[8];
         load8(dxp + (size_t)rows[0] * d + c, out);
@@ -595,6 +682,15 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
             load8(w_router + (size_t)e[j] * d + c, wv);
 #pragma unroll
             for (int u = 0; u < 8; ++u) out[u] = fmaf(dzv[j], wv[u], out[u]);
+        }
+        if (aux_scale != 0.f) {
+            for (int m = 0; m < N; ++m) {
+                const float pm = expf(zt[m] - zmax) * inv_den;
+                const float dza = aux_scale * pm * ((float)counts_slot[m] * inv_T - fp);
+                load8(w_router + (size_t)m * d + c, wv);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) out[u] = fmaf(dza, wv[u], out[u]);
+            }
         }
         store8(dx + (size_t)t * d + c, out);
     }
@@ -609,16 +705,21 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
 template <typename T>
 __global__ void __launch_bounds__(256)
 router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int *__restrict__ topk_idx,
-                  const float *__restrict__ dz, float *__restrict__ dwr_partial)
+                  const float *__restrict__ dz, float *__restrict__ dwr_partial, const float *__restrict__ logits,
+                  const int *__restrict__ counts_slot, float aux_scale)
 {
     constexpr int CPT = (sizeof(T) == 2) ? 2 : 1;        // columns per thread: one 4-byte load either way
     __shared__ float dzs[kRouterBwdTokB][8];
     __shared__ int idxs[kRouterBwdTokB][2];
     __shared__ float dzk[kRouterBwdTokB][2];
+    __shared__ float smax[kRouterBwdTokB], sinv[kRouterBwdTokB], sfp[kRouterBwdTokB];
     const int tid = threadIdx.x;
     const int t0 = blockIdx.x * kRouterBwdTokB;
     const int c = (blockIdx.y * 256 + tid) * CPT;
     const int ntok = min(kRouterBwdTokB, Ttok - t0);
+    const float inv_T = 1.0f / (float)Ttok;
+    if (aux_scale != 0.f && tid < ntok)
+        token_softmax_stats(logits + (size_t)(t0 + tid) * N, counts_slot, N, inv_T, smax[tid], sinv[tid], sfp[tid]);
     for (int i = tid; i < kRouterBwdTokB * 2; i += 256) {
         const int tl = i >> 1, j = i & 1;
         const bool ok = tl < ntok && j < k;
@@ -632,6 +733,10 @@ router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const 
             float v = 0.f;
             if (idxs[tl][0] == e) v = dzk[tl][0];
             if (idxs[tl][1] == e) v = dzk[tl][1];
+            if (aux_scale != 0.f && tl < ntok && e < N) {
+                const float pm = expf(logits[(size_t)(t0 + tl) * N + e] - smax[tl]) * sinv[tl];
+                v += aux_scale * pm * ((float)counts_slot[e] * inv_T - sfp[tl]);
+            }
             dzs[tl][i & 7] = v;
         }
         __syncthreads();
@@ -702,7 +807,7 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             kern<<<nblk, kRouterMmaThreads, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
-                                         p.topk_idx, p.topk_gate, p.block_counts);
+                                         p.topk_idx, p.topk_gate, p.block_counts, p.logits);
             MODSE_LAUNCH_CHECK();
             return cudaSuccess;
         }
@@ -717,13 +822,13 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<nblk, 256, smem, s>>>((const float *)x, (const float *)w_router, T, m.d, m.N, m.k, p.topk_idx,
-                                     p.topk_gate, p.block_counts, w_in_smem);
+                                     p.topk_gate, p.block_counts, p.logits, w_in_smem);
     } else {
         auto kern = router_kernel<__nv_bfloat16>;
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<nblk, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
-                                     p.topk_idx, p.topk_gate, p.block_counts, w_in_smem);
+                                     p.topk_idx, p.topk_gate, p.block_counts, p.logits, w_in_smem);
     }
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
@@ -789,32 +894,44 @@ cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *
 
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
                               int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
-                              cudaStream_t s, int *launches)
+                              float aux_scale, cudaStream_t s, int *launches)
 {
     const int grid_dx = (T + 7) / 8;
     const float *dxp = (const float *)p.dxp;
     if (dt == MODSE_F32)
         router_dx_kernel<float, float><<<grid_dx, 256, 0, s>>>((const float *)w_router, dxp, T, m.d, m.k, p.topk_idx,
-                                                               p.topk_gate, p.prow_of, p.dg, p.dz, (float *)dx);
+                                                               p.topk_gate, p.prow_of, p.dg, p.dz, (float *)dx, m.N, p.logits,
+                                                               p.counts_slot, aux_scale);
     else if (out_f32)
         router_dx_kernel<__nv_bfloat16, float><<<grid_dx, 256, 0, s>>>((const __nv_bfloat16 *)w_router, dxp, T, m.d,
                                                                        m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg,
-                                                                       p.dz, (float *)dx);
+                                                                       p.dz, (float *)dx, m.N, p.logits, p.counts_slot,
+                                                                       aux_scale);
     else
         router_dx_kernel<__nv_bfloat16, __nv_bfloat16><<<grid_dx, 256, 0, s>>>(
             (const __nv_bfloat16 *)w_router, dxp, T, m.d, m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz,
-            (__nv_bfloat16 *)dx);
+            (__nv_bfloat16 *)dx, m.N, p.logits, p.counts_slot, aux_scale);
     MODSE_LAUNCH_CHECK();
     dim3 grid(nblk_bwd, dt == MODSE_F32 ? (m.d + 255) / 256 : (m.d + 511) / 512);
     if (dt == MODSE_F32)
         router_dwr_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.topk_idx, p.dz,
-                                                      p.dwr_partial);
+                                                      p.dwr_partial, p.logits, p.counts_slot, aux_scale);
     else
         router_dwr_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k, p.topk_idx,
-                                                              p.dz, p.dwr_partial);
+                                                              p.dz, p.dwr_partial, p.logits, p.counts_slot, aux_scale);
     MODSE_LAUNCH_CHECK();
     const int n = m.N * m.d;
     reduce_dwr_kernel<<<(n + 255) / 256, 256, 0, s>>>(p.dwr_partial, nblk_bwd, n, dw_router);
+    MODSE_LAUNCH_CHECK();
+    return cudaSuccess;
+}
+
+cudaError_t launch_aux_loss(const LayerMeta &m, int T, int nblk_bwd, const WsPtrs &p, float alpha, float *loss,
+                            float *f, float *P, cudaStream_t s, int *launches)
+{
+    aux_partial_kernel<<<nblk_bwd, 128, 0, s>>>(p.logits, T, m.N, p.aux_partial);
+    MODSE_LAUNCH_CHECK();
+    aux_final_kernel<<<1, 256, 0, s>>>(p.aux_partial, nblk_bwd, p.counts_slot, T, m.N, alpha, loss, f, P);
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
 }
