@@ -34,6 +34,28 @@ from paper_2409_12210_b200 import inputs as I  # noqa: E402
 METRIC = "modse_layer_fwd_bwd_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+# profiles/tc_grouped_gemm_train_16k_ncu_full.md; valid only for that workload and for the kernel source it was
+# taken from (first 16 hex digits of the SHA-256 of csrc/tc_gemm.cu), otherwise "traffic" is reported as null.
+NCU_TRAFFIC = {
+    "workload": "train_16k", "tc_gemm_sha256_16": "73d4134c4ed1aaf9",
+    "bytes_per_launch": {"upgate_gemm_swiglu": 1.590e9, "down_gemm": 0.964e9, "down_dgrad_swiglu_bwd": 1.981e9,
+                         "down_wgrad": 0.751e9, "upgate_dgrad": 1.835e9, "upgate_wgrad": 1.326e9},
+}
+
+
+def ncu_traffic(stage: str, workload: str):
+    import hashlib
+    try:
+        src = os.path.join(ROOT, "paper_2409_12210_b200", "csrc", "tc_gemm.cu")
+        digest = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    except OSError:
+        return None
+    if workload != NCU_TRAFFIC["workload"] or digest != NCU_TRAFFIC["tc_gemm_sha256_16"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"].get(stage)
+
+
 STAGE_BOUND = ["hbm", "hbm", "hbm", "tensor", "tensor", "hbm", "hbm", "tensor", "tensor", "tensor", "tensor", "hbm"]
 
 
@@ -355,7 +377,8 @@ def main():
     dom = max(stages, key=lambda s: s["ms"])
     roofline = {"kernel": dom["stage"], "bound": dom["bound"], "achieved": dom["achieved"],
                 "peak": pk["bf16_tflops_sustained"] if dom["bound"] == "tensor" else pk["hbm_gbs"],
-                "unit": dom["unit"], "frac": dom["frac"], "traffic": None, "peak_source": f"of {pk_src}",
+                "unit": dom["unit"], "frac": dom["frac"], "traffic": ncu_traffic(dom["stage"], cfg.name),
+                "traffic_unit": "bytes per launch (ncu dram read + write)", "peak_source": f"of {pk_src}",
                 "ms_per_launch": dom["ms"]}
 
     cpu = None
