@@ -53,6 +53,12 @@ CONFIGS = {
     "train_16k": LayerConfig("train_16k", "bf16", 2048, WIDTHS_700M, 2, 16384, weight_std=0.02),
     "train_16k_equal": LayerConfig("train_16k_equal", "bf16", 2048, WIDTHS_EQUAL, 2, 16384, weight_std=0.02),
     "train_64k": LayerConfig("train_64k", "bf16", 2048, WIDTHS_700M, 2, 65536, weight_std=0.02),
+    # size-diversity sweep at a fixed pair sum of 11264 (ratio 1 = train_16k_equal, ratio 3 = train_16k)
+    "train_16k_ratio2": LayerConfig("train_16k_ratio2", "bf16", 2048, WIDTHS_RATIO2, 2, 16384, weight_std=0.02),
+    "train_16k_ratio4": LayerConfig("train_16k_ratio4", "bf16", 2048, WIDTHS_RATIO4, 2, 16384, weight_std=0.02),
+    # the paper's own expert widths (Table 2): ratio 9 at width 2048, and the 300M x 8 model at width 1536
+    "table2_700m": LayerConfig("table2_700m", "bf16", 2048, WIDTHS_TABLE2_700M, 2, 16384, weight_std=0.02),
+    "table2_300m": LayerConfig("table2_300m", "bf16", 1536, WIDTHS_TABLE2_300M, 2, 16384, weight_std=0.02),
     "train_16k_skew": LayerConfig("train_16k_skew", "bf16", 2048, WIDTHS_700M, 2, 16384, weight_std=0.02,
                                   router_bias=ZIPF_ROUTER_BIAS),
     "train_16k_equal_skew": LayerConfig("train_16k_equal_skew", "bf16", 2048, WIDTHS_EQUAL, 2, 16384,

@@ -73,7 +73,7 @@ def compare(gpu, ora, cfg, backward, discount):
     return errs
 
 
-@pytest.mark.parametrize("name", ["fwd_8k", "train_16k", "train_16k_skew"])
+@pytest.mark.parametrize("name", ["fwd_8k", "train_16k", "train_16k_skew", "table2_700m", "table2_300m"])
 def test_full_size_sampled_parity(name):
     cfg = I.CONFIGS[name]
     inp, n_redrawn = H.screened(cfg)
