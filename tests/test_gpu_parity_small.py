@@ -136,3 +136,58 @@ def test_bf16_degenerate_and_ragged_shapes(T, k, widths, d):
     # dz = g (dg - sum g dg) cancels; over one or two tokens its RMS is that of a few numbers,
     # so dz and dW_router = dz^T x keep the max bound above and are left out of the RMS one
     H.check_rms(gpu, ora, RMS_TOL_BF16, skip=("dz", "dw_router") if T < 64 else ())
+
+
+def test_bf16_single_expert_top1_is_a_dense_swiglu_ffn():
+    cfg = I.LayerConfig("bf16_dense", "bf16", 256, (448,), 1, 500, seed=9, weight_std=0.05)
+    inp = I.generate(cfg)
+    gpu = H.run_gpu(inp, True, out_f32=True)
+    ora = H.run_oracle(inp, True)
+    H.check_all(inp, gpu, ora, TOL_BF16)
+    assert np.all(gpu["routing"]["topk_gate"] == 1.0) and np.all(gpu["dw_router"] == 0.0)
+
+
+def test_bf16_empty_expert_gets_zero_weight_gradients():
+    inp, _ = H.screened(SMALL_BF16)
+    inp.x = np.abs(inp.x); inp.w_router = np.abs(inp.w_router); inp.w_router[2] = -inp.w_router[2]
+    gpu = H.run_gpu(inp, True, out_f32=True)
+    ora = H.run_oracle(inp, True)
+    assert ora["rt"].counts[2] == 0
+    # all-positive inputs route very unevenly here, so the experts' gradient magnitudes differ a lot:
+    # the pooled max bound is kept for the token-major tensors, the RMS bound for all
+    H.check_all(inp, gpu, ora, TOL_BF16, only=("y", "dx", "dg", "dz", "dw_router"))
+    H.check_rms(gpu, ora, RMS_TOL_BF16)
+    h0, h1 = sum(SMALL_BF16.ffn_sizes[:2]), sum(SMALL_BF16.ffn_sizes[:3])
+    assert np.all(gpu["dw_gate"][h0:h1] == 0) and np.all(gpu["dw_up"][h0:h1] == 0)
+    assert np.all(gpu["dw_down"][:, h0:h1] == 0)
+
+
+@pytest.mark.parametrize("n_experts", [16, 40])
+def test_bf16_many_experts(n_experts):
+    # 16 experts: two 8-expert tiles in the tensor-core router; 40: the general fp32-FMA router
+    rng = np.random.default_rng(n_experts)
+    widths = tuple(int(w) for w in rng.choice([64, 128, 192, 256], n_experts))
+    cfg = I.LayerConfig(f"bf16_N{n_experts}", "bf16", 256, widths, 2, 3000, seed=n_experts, weight_std=0.05)
+    inp, _ = H.screened(cfg)
+    gpu = H.run_gpu(inp, True, out_f32=True)
+    ora = H.run_oracle(inp, True)
+    H.check_all(inp, gpu, ora, TOL_BF16, only=("y", "dx", "dg", "dz", "dw_router"))
+    H.check_rms(gpu, ora, RMS_TOL_BF16)
+
+
+def test_bf16_results_are_bitwise_reproducible_and_independent_of_tile_shape():
+    from paper_2409_12210_b200 import binding as B
+    inp, _ = H.screened(SMALL_BF16)
+    a = H.run_gpu(inp, True)
+    b = H.run_gpu(inp, True)
+    B.debug_set_pair_kernels(0)                     # 128-row tiles everywhere
+    try:
+        c = H.run_gpu(inp, True)
+        B.debug_set_pair_kernels(63)                # two-SM tiles everywhere
+        e = H.run_gpu(inp, True)
+    finally:
+        B.debug_set_pair_kernels((2 | 8 | 16 | 32) << 8)   # the library's default
+    for k in ("y", "dx", "dw_router", "dw_gate", "dw_up", "dw_down", "dg", "dz"):
+        assert np.array_equal(a[k], b[k]), k
+        assert np.array_equal(a[k], c[k]), k
+        assert np.array_equal(a[k], e[k]), k
