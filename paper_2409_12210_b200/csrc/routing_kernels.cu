@@ -203,7 +203,7 @@ constexpr int kRouterKSplit = 4;     // warps per 16-token group, each summing a
 constexpr int kRouterMmaThreads = 4 * kRouterKSplit * 32;
 
 template <int NT>
-__global__ void __launch_bounds__(kRouterMmaThreads)
+__global__ void __launch_bounds__(kRouterMmaThreads, 2)      // two 512-thread blocks per SM: at most 64 registers
 router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w_router, int Ttok, int d,
                   int N, int k, int *__restrict__ topk_idx, float *__restrict__ topk_gate,
                   int *__restrict__ block_counts, float *__restrict__ logits)
@@ -248,16 +248,6 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
     for (int it0 = 0; it0 < niter; it0 += UB) {
-        uint4 ca[UB], cb[UB];
-#pragma unroll
-        for (int u = 0; u < UB; ++u) { ca[u] = xa[u]; cb[u] = xb[u]; }
-#pragma unroll
-        for (int u = 0; u < UB; ++u) {
-            const int it = it0 + UB + u;
-            const int c0 = cbeg + it * 32;
-            xa[u] = (v0 && it < niter) ? x0[c0 >> 3] : za;
-            xb[u] = (v1 && it < niter) ? x1[c0 >> 3] : za;
-        }
 #pragma unroll
         for (int u = 0; u < UB; ++u) {
             const int c0 = cbeg + (it0 + u) * 32;
@@ -265,10 +255,15 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const uint4 w = *reinterpret_cast<const uint4 *>(wsm + (size_t)(nt * 8 + g) * ldw + c0 + tq * 8);
-                    mma_bf16_16816(acc[nt], ca[u].x, cb[u].x, ca[u].y, cb[u].y, w.x, w.y);
-                    mma_bf16_16816(acc[nt], ca[u].z, cb[u].z, ca[u].w, cb[u].w, w.z, w.w);
+                    mma_bf16_16816(acc[nt], xa[u].x, xb[u].x, xa[u].y, xb[u].y, w.x, w.y);
+                    mma_bf16_16816(acc[nt], xa[u].z, xb[u].z, xa[u].w, xb[u].w, w.z, w.w);
                 }
             }
+            // refill this slot with the chunk UB iterations ahead as soon as it has been consumed
+            const int it = it0 + UB + u;
+            const int cn = cbeg + it * 32;
+            xa[u] = (v0 && it < niter) ? x0[cn >> 3] : za;
+            xb[u] = (v1 && it < niter) ? x1[cn >> 3] : za;
         }
     }
     // the other warps hand their partial logits to the first warp of the same token group,
