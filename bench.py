@@ -216,10 +216,15 @@ def main():
     ap.add_argument("--workload", default="train_16k", choices=sorted(I.CONFIGS))
     ap.add_argument("--cpu-tokens", type=int, default=64, help="tokens of the CPU baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tokens", type=int, default=None, help="override the workload's token count")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="layer-stack sweep: a step runs this many independent layers (own weights, x and dY each)")
     ap.add_argument("--pair-mask", type=int, default=None,
                     help="tuning: which grouped products use the two-SM kernel (bit per product)")
     args = ap.parse_args()
     cfg = I.CONFIGS[args.workload]
+    if args.tokens is not None:
+        cfg = I.with_tokens(cfg, args.tokens)
     if args.impl == "reference":
         run_reference(args, cfg)
         return
@@ -248,6 +253,15 @@ def main():
     wr, wg, wu, wd = B.pack_weights(inp, dev)
     x = torch.from_numpy(inp.x).to(dev, dt)
     dy = torch.from_numpy(inp.dy).to(dev, dt)
+    # layer-stack mode: layers 1.. get their own seeded weights, tokens and upstream gradients, drawn on the
+    # device with the same distributions (layer 0 is the workload's own tensors); no data flows between layers
+    L = max(1, args.layers)
+    extra = []
+    for l in range(1, L):
+        gen = torch.Generator(device=dev).manual_seed(cfg.seed + 1000 + l)
+        rn = lambda ref, std: (torch.randn(ref.shape, generator=gen, device=dev, dtype=torch.float32) * std).to(dt)
+        wstd = cfg.weight_std if cfg.weight_std is not None else d ** -0.5
+        extra.append((rn(wr, wstd), rn(wg, wstd), rn(wu, wstd), rn(wd, wstd), rn(x, 1.0), rn(dy, 1.0)))
     y, dx = torch.empty_like(x), torch.empty_like(x)
     dwr = torch.empty(wr.shape, dtype=torch.float32, device=dev)
     dwg, dwu, dwd = torch.empty_like(wg), torch.empty_like(wu), torch.empty_like(wd)
@@ -262,6 +276,12 @@ def main():
         if do_bwd:
             layer.backward(wr, wg, wu, wd, xb, dyb, dxb, dwr, dwg, dwu, dwd, ws)
             n += layer.last_launch_count()
+        for (wr_l, wg_l, wu_l, wd_l, x_l, dy_l) in extra:
+            layer.forward(wr_l, wg_l, wu_l, wd_l, x_l, yb, ws, do_bwd)
+            n += layer.last_launch_count()
+            if do_bwd:
+                layer.backward(wr_l, wg_l, wu_l, wd_l, x_l, dy_l, dxb, dwr, dwg, dwu, dwd, ws)
+                n += layer.last_launch_count()
         return n
 
     def sync_all():
@@ -280,7 +300,7 @@ def main():
 
     # ---- device-resident timing: K steps between two events, stages bracketed by the library's own events ----
     sampler = ClockSampler(local_rank)
-    n_calls = K * (2 if do_bwd else 1)
+    n_calls = K * L * (2 if do_bwd else 1)
     layer.stage_timing_begin(n_calls)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
@@ -359,7 +379,7 @@ def main():
     # ---- roofline of every stage, and of the dominant one ----
     pk, pk_src = peaks()
     fwd_flops, bwd_flops, _ = expert_flops(counts, cfg)
-    flops_step = fwd_flops + (bwd_flops if do_bwd else 0.0)
+    flops_step = L * (fwd_flops + (bwd_flops if do_bwd else 0.0))     # layers 1.. route near-uniformly like layer 0
     work = stage_work(counts, cfg)
     stages = []
     for i in range(B.N_STAGES):
@@ -392,7 +412,8 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "d_model": d, "ffn_sizes": list(cfg.ffn_sizes), "top_k": cfg.top_k,
-                   "n_tokens": T, "pass": "fwd+bwd" if do_bwd else "fwd", "parallelism": f"replicas x{world}",
+                   "n_tokens": T, "layers": L,
+                   "e2e_copies": "x, dY in and y, dx out of layer 0" if L > 1 else "x, dY in; y, dx out", "pass": "fwd+bwd" if do_bwd else "fwd", "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (weights 554 MB, activations > 126 MB per step)"},
         "tflops": flops_step / (ms_step * 1e-3) / 1e12,
         "tflops_frac_of_sustained_peak": flops_step / (ms_step * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
