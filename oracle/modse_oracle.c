@@ -472,3 +472,123 @@ int modse_oracle_aux_loss(int T, int N, const double *z, double alpha,
     free(f); free(P); free(p);
     return 0;
 }
+
+/* ------------------------------------------------------------------ */
+/* Sec. 2, Eq. 2 (second term), Eq. 4-5 of the preliminaries:           */
+/*   H(x)_i = (x W_g)_i + RMSNorm(f((x W_n)_i)),  f = Softplus,          */
+/*   RMSNorm(v)_i = gamma v_i / sqrt(mean_j v_j^2 + eps)                 */
+/* read as: u = x W_n (one entry per expert), s = softplus(u), the RMS  */
+/* taken over the N expert entries of the token, gamma a scalar.        */
+/* noise_term writes r[t,i] (and u, s if wanted) for every token.       */
+/* ------------------------------------------------------------------ */
+static double softplus(double u) { return u > 0 ? u + log1p(exp(-u)) : log1p(exp(u)); }
+
+int modse_oracle_noise_term(int T, int d, int N, const double *x, const double *w_noise,
+                            double gamma, double eps, double *r, double *u_out)
+{
+    if (T < 0 || d < 1 || N < 1) return -1;
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        double ms = 0.0;
+        for (int i = 0; i < N; ++i) {
+            double u = dot(x + (size_t)t * d, w_noise + (size_t)i * d, d);
+            if (u_out) u_out[(size_t)t * N + i] = u;
+            double s = softplus(u);
+            r[(size_t)t * N + i] = s;
+            ms += s * s;
+        }
+        double inv = gamma / sqrt(ms / N + eps);
+        for (int i = 0; i < N; ++i) r[(size_t)t * N + i] *= inv;
+    }
+    return 0;
+}
+
+/* Gradient of the noise term given dz = dL/dH (all N entries per token):
+ *   s = softplus(u), q = sqrt(mean s^2 + eps), r = gamma s / q
+ *   dgamma += sum_i dz_i s_i / q
+ *   ds_i = gamma (dz_i / q - s_i (sum_j dz_j s_j) / (N q^3))
+ *   du_i = ds_i sigmoid(u_i);  dW_n += du^T x;  dx_add = du W_n          */
+int modse_oracle_noise_backward(int T, int d, int N, const double *x, const double *w_noise,
+                                double gamma, double eps, const double *dz,
+                                double *dx_add, double *dw_noise, double *dgamma)
+{
+    if (T < 0 || d < 1 || N < 1) return -1;
+    memset(dw_noise, 0, sizeof(double) * (size_t)N * d);
+    double dg = 0.0;
+    double *s = (double *)malloc(sizeof(double) * 3 * (size_t)N);
+    if (!s) return -3;
+    double *u = s + N, *du = u + N;
+    for (int t = 0; t < T; ++t) {
+        const double *xt = x + (size_t)t * d, *dzt = dz + (size_t)t * N;
+        double ms = 0.0, dzs = 0.0;
+        for (int i = 0; i < N; ++i) {
+            u[i] = dot(xt, w_noise + (size_t)i * d, d);
+            s[i] = softplus(u[i]);
+            ms += s[i] * s[i];
+            dzs += dzt[i] * s[i];
+        }
+        double q = sqrt(ms / N + eps);
+        dg += dzs / q;
+        for (int i = 0; i < N; ++i) {
+            double ds = gamma * (dzt[i] / q - s[i] * dzs / (N * q * q * q));
+            du[i] = ds * sigmoid(u[i]);
+        }
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int i = 0; i < N; ++i) {
+                acc += du[i] * w_noise[(size_t)i * d + c];
+                dw_noise[(size_t)i * d + c] += du[i] * xt[c];
+            }
+            dx_add[(size_t)t * d + c] = acc;
+        }
+    }
+    *dgamma = dg;
+    free(s);
+    return 0;
+}
+
+/* Routing tables from given logits z [T,N] (top-k, gates, counts, permutation): the second
+ * half of modse_oracle_route, for logits that carry the noise term.                        */
+int modse_oracle_route_from_logits(int T, int N, int k, const double *z, int *topk_idx,
+                                   double *topk_gate, int *counts, int *counts_slot, int *offsets,
+                                   int *row_of, int *token_of)
+{
+    if (T < 0 || N < 1 || k < 1 || k > N) return -1;
+    for (int t = 0; t < T; ++t) {
+        const double *zt = z + (size_t)t * N;
+        for (int j = 0; j < k; ++j) {
+            int best = -1;
+            for (int i = 0; i < N; ++i) {
+                int taken = 0;
+                for (int jj = 0; jj < j; ++jj) if (topk_idx[(size_t)t * k + jj] == i) taken = 1;
+                if (taken) continue;
+                if (best < 0 || zt[i] > zt[best]) best = i;
+            }
+            topk_idx[(size_t)t * k + j] = best;
+        }
+        double m = zt[topk_idx[(size_t)t * k]], den = 0.0;
+        for (int j = 0; j < k; ++j) den += exp(zt[topk_idx[(size_t)t * k + j]] - m);
+        for (int j = 0; j < k; ++j) topk_gate[(size_t)t * k + j] = exp(zt[topk_idx[(size_t)t * k + j]] - m) / den;
+    }
+    for (int e = 0; e < N; ++e) counts[e] = 0;
+    for (int i = 0; i < k * N; ++i) counts_slot[i] = 0;
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < k; ++j) {
+            int e = topk_idx[(size_t)t * k + j];
+            counts[e] += 1;
+            counts_slot[j * N + e] += 1;
+        }
+    offsets[0] = 0;
+    for (int e = 0; e < N; ++e) offsets[e + 1] = offsets[e] + counts[e];
+    int *fill = (int *)calloc((size_t)N, sizeof(int));
+    if (!fill) return -3;
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < k; ++j) {
+            int e = topk_idx[(size_t)t * k + j];
+            int row = offsets[e] + fill[e]++;
+            row_of[(size_t)t * k + j] = row;
+            token_of[row] = t;
+        }
+    free(fill);
+    return 0;
+}

@@ -104,6 +104,22 @@ int modse_oracle_backward(int T, int d, int N, int k, const int *h,
 int modse_oracle_aux_loss(int T, int N, const double *z, double alpha,
                           double *loss, double *f, double *P, double *dz_aux);
 
+/* Second term of H(x) (Sec. 2, Eq. 2 with Eq. 4-5): r[t,i] = RMSNorm(Softplus(x W_n))_i with the
+ * RMS taken over the N expert entries of token t and a scalar gamma; u_out [T,N] (may be NULL)
+ * receives x W_n.                                                                            */
+int modse_oracle_noise_term(int T, int d, int N, const double *x, const double *w_noise,
+                            double gamma, double eps, double *r, double *u_out);
+
+/* Its gradient for dz = dL/dH [T,N]: dx_add [T,d] (to be added to dx), dw_noise [N,d], dgamma. */
+int modse_oracle_noise_backward(int T, int d, int N, const double *x, const double *w_noise,
+                                double gamma, double eps, const double *dz,
+                                double *dx_add, double *dw_noise, double *dgamma);
+
+/* Top-k, gates and permutation tables from given logits z [T,N] (same rules as modse_oracle_route). */
+int modse_oracle_route_from_logits(int T, int N, int k, const double *z, int *topk_idx,
+                                   double *topk_gate, int *counts, int *counts_slot, int *offsets,
+                                   int *row_of, int *token_of);
+
 int modse_oracle_num_threads(void);
 
 #ifdef __cplusplus

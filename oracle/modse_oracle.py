@@ -204,6 +204,43 @@ def aux_loss(z, alpha: float):
     return loss.value, f, P, dz
 
 
+def noise_term(x, w_noise, gamma: float, eps: float):
+    """(r [T,N], u [T,N]): r = RMSNorm(Softplus(x W_n)) over the expert entries, u = x W_n."""
+    x = _f64(x); w_noise = _f64(w_noise)
+    T, d = x.shape
+    N = w_noise.shape[0]
+    r = np.empty((T, N)); u = np.empty((T, N))
+    rc = lib().modse_oracle_noise_term(T, d, N, _d(x), _d(w_noise), ctypes.c_double(gamma), ctypes.c_double(eps),
+                                       _d(r), _d(u))
+    _check(rc, "noise_term")
+    return r, u
+
+
+def noise_backward(x, w_noise, gamma: float, eps: float, dz):
+    """(dx_add [T,d], dw_noise [N,d], dgamma) for dz = dL/dH [T,N]."""
+    x = _f64(x); w_noise = _f64(w_noise); dz = _f64(dz)
+    T, d = x.shape
+    N = w_noise.shape[0]
+    dx = np.empty((T, d)); dw = np.empty((N, d)); dg = ctypes.c_double(0.0)
+    rc = lib().modse_oracle_noise_backward(T, d, N, _d(x), _d(w_noise), ctypes.c_double(gamma),
+                                           ctypes.c_double(eps), _d(dz), _d(dx), _d(dw), ctypes.byref(dg))
+    _check(rc, "noise_backward")
+    return dx, dw, dg.value
+
+
+def route_from_logits(z, k: int) -> Routing:
+    z = _f64(z)
+    T, N = z.shape
+    idx = np.empty((T, k), np.int32); gate = np.empty((T, k))
+    counts = np.empty(N, np.int32); cs = np.empty((k, N), np.int32)
+    offsets = np.empty(N + 1, np.int32); row_of = np.empty((T, k), np.int32)
+    token_of = np.empty(k * T, np.int32)
+    rc = lib().modse_oracle_route_from_logits(T, N, k, _d(z), _i(idx), _d(gate), _i(counts), _i(cs), _i(offsets),
+                                              _i(row_of), _i(token_of))
+    _check(rc, "route_from_logits")
+    return Routing(z, idx, gate, counts, cs, offsets, row_of, token_of)
+
+
 def routing_margin(z: np.ndarray, k: int) -> np.ndarray:
     """Smallest gap between consecutive logits among the k+1 largest of each
     token: the distance of the top-k decision (and its order) from a flip."""
