@@ -177,6 +177,29 @@ modse_status_t modse_set_aux_loss(modse_layer_t *layer, float alpha);
  * accumulation over micro-batches in fp32.  No effect on fp32 layers.        */
 modse_status_t modse_set_output_f32(modse_layer_t *layer, int on);
 
+/* Second term of the router logits (Sec. 2, Eq. 2 with the RMSNorm and Softplus
+ * definitions that follow it):
+ *   H(x)_i = (x W_g)_i + RMSNorm(Softplus((x W_n)_i)),
+ *   RMSNorm(v)_i = gamma v_i / sqrt(mean_j v_j^2 + eps),
+ * read as: W_n is a second [N,d] router matrix, the mean runs over the N expert
+ * entries of a token, gamma is one learnable scalar.  The term is a function of
+ * x alone (the paper draws no random number here), so it is simply part of the
+ * logits that top-k, the gates, the auxiliary loss and the backward pass see.
+ *
+ * modse_set_noise_gate: w_noise is a DEVICE pointer to [N,d] in the layer's
+ * dtype, 16-byte aligned, borrowed until it is replaced (it must stay valid for
+ * every later forward/backward); NULL switches the term off (the default).
+ * gamma any finite value, eps >= 0.
+ * modse_set_noise_grads: where modse_backward writes dW_n ([N,d] fp32, device,
+ * 16-byte aligned) and dgamma (one fp32, device); both overwritten.  Required
+ * before a backward whose forward ran with the term on (else
+ * MODSE_ERR_INVALID_ARG); a backward whose on/off state differs from its
+ * forward's returns MODSE_ERR_STATE.
+ * dx and the router gradients then include the term's contribution; every sum
+ * has a fixed order as elsewhere.                                            */
+modse_status_t modse_set_noise_gate(modse_layer_t *layer, const void *w_noise, float gamma, float eps);
+modse_status_t modse_set_noise_grads(modse_layer_t *layer, float *dw_noise, float *dgamma);
+
 /* Routing only, with no device allocation by anyone.  (The paper has no
  * counterpart: this is a packaging variant of the router stage of Eq. 2-3.)
  *

@@ -91,6 +91,10 @@ def load():
     lib.modse_aux_loss.argtypes = [vp, vp, ci, ctypes.c_float, vp, vp, vp, vp]
     lib.modse_set_aux_loss.restype = ci
     lib.modse_set_aux_loss.argtypes = [vp, ctypes.c_float]
+    lib.modse_set_noise_gate.restype = ci
+    lib.modse_set_noise_gate.argtypes = [vp, vp, ctypes.c_float, ctypes.c_float]
+    lib.modse_set_noise_grads.restype = ci
+    lib.modse_set_noise_grads.argtypes = [vp, vp, vp]
     lib.modse_set_output_f32.restype = ci
     lib.modse_set_output_f32.argtypes = [vp, ci]
     lib.modse_stage_timing_begin.restype = ci
@@ -277,6 +281,23 @@ class ModseLayer:
         if st != MODSE_OK:
             raise ModseError(st, "modse_aux_loss")
         return loss, f, P
+
+    def set_noise_gate(self, w_noise, gamma: float = 0.0, eps: float = 0.0) -> None:
+        """Second term of the router logits (Eq. 2): w_noise is a device tensor [N,d] in the layer's dtype
+        that the caller keeps alive, or None to switch the term off."""
+        self._w_noise = w_noise
+        st = load().modse_set_noise_gate(self._h, w_noise.data_ptr() if w_noise is not None else None,
+                                         float(gamma), float(eps))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_set_noise_gate")
+
+    def set_noise_grads(self, dw_noise, dgamma) -> None:
+        """Device tensors that backward fills: dw_noise [N,d] fp32, dgamma [1] fp32."""
+        self._noise_grads = (dw_noise, dgamma)
+        st = load().modse_set_noise_grads(self._h, dw_noise.data_ptr() if dw_noise is not None else None,
+                                          dgamma.data_ptr() if dgamma is not None else None)
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_set_noise_grads")
 
     def set_output_f32(self, on: bool) -> None:
         st = load().modse_set_output_f32(self._h, int(bool(on)))

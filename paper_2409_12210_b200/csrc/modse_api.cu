@@ -16,9 +16,11 @@ struct modse_layer {
     int fwd_tokens = -1;
     int fwd_dtype = -1;
     int fwd_saved = 0;
+    int fwd_noise = 0;            // the last forward's logits carried the second term
     int last_launches = 0;
     float aux_alpha = 0.f;        // coefficient of the auxiliary load-balance loss added to the objective in backward
     int out_f32 = 0;              // bf16 layers: write y, dx and expert weight gradients as fp32
+    modse::NoiseGate noise;       // second term of the router logits (borrowed device pointers)
     modse::TcPlan tc;             // device facts of the bf16 path
     // optional per-stage device timing: events [call][stage][start/stop]
     std::vector<cudaEvent_t> ev;
@@ -61,6 +63,7 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
     L.block_counts = take((size_t)L.nblk * m.k * N * 4);
     L.logits = take((size_t)T * N * 4);
     L.aux_partial = take((size_t)L.nblk_bwd * N * 4);
+    L.noise_u = take((size_t)T * N * 4);
     L.xp = take((size_t)L.Pmax * m.d * esz);
     L.hm = take(L.hb * esz);
     L.o = take((size_t)L.Pmax * m.d * 4);     // fp32 for every layer type
@@ -69,6 +72,8 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
         L.b_pre = take(L.hb * esz);
         L.dg = take(kT * 4);
         L.dz = take(kT * 4);
+        L.du = take((size_t)T * N * 4);
+        L.dgamma_partial = take((size_t)L.nblk_bwd * 4);
         L.dwr_partial = take((size_t)L.nblk_bwd * N * m.d * 4);
         L.dyp = take((size_t)L.Pmax * m.d * esz);
         L.da = take(L.hb * esz);
@@ -103,6 +108,9 @@ WsPtrs carve(void *ws, const WsLayout &L)
     p.block_counts = (int *)(b + L.block_counts);
     p.logits = (float *)(b + L.logits);
     p.aux_partial = (float *)(b + L.aux_partial);
+    p.noise_u = (float *)(b + L.noise_u);
+    p.du = (float *)(b + L.du);
+    p.dgamma_partial = (float *)(b + L.dgamma_partial);
     p.dg = (float *)(b + L.dg);
     p.dz = (float *)(b + L.dz);
     p.dwr_partial = (float *)(b + L.dwr_partial);
@@ -296,7 +304,7 @@ modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const mo
 
     StageTimer tm(layer, s);
     MODSE_CUDA(cudaMemsetAsync(p.status, 0, 64, s));
-    MODSE_STAGE(tm, 0, launch_router(dtype, m, x, weights->w_router, n_tokens, p, s, &launches));
+    MODSE_STAGE(tm, 0, launch_router(dtype, m, x, weights->w_router, n_tokens, p, layer->noise, s, &launches));
     MODSE_STAGE(tm, 1, launch_rank(m, n_tokens, L.Pmax, p, s, &launches));
     MODSE_STAGE(tm, 2, launch_permute(dtype, m, x, n_tokens, p, s, &launches));
     if (dtype == MODSE_F32 || tc_force_simt()) {
@@ -323,6 +331,7 @@ modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const mo
     layer->fwd_tokens = n_tokens;
     layer->fwd_dtype = (int)dtype;
     layer->fwd_saved = save ? 1 : 0;
+    layer->fwd_noise = layer->noise.w_noise != nullptr ? 1 : 0;
     layer->last_launches = launches;
     return MODSE_OK;
 }
@@ -341,6 +350,9 @@ modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const m
     if (layer->fwd_ws != workspace || layer->fwd_tokens != n_tokens || layer->fwd_dtype != (int)dtype ||
         !layer->fwd_saved)
         return MODSE_ERR_STATE;
+    if ((layer->noise.w_noise != nullptr) != (layer->fwd_noise != 0)) return MODSE_ERR_STATE;
+    if (layer->noise.w_noise != nullptr && (!aligned16(layer->noise.dw_noise) || layer->noise.dgamma == nullptr))
+        return MODSE_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const LayerMeta &m = layer->meta;
     const WsLayout L = make_layout(m, layer->h_desc.data(), dtype == MODSE_F32 ? 4 : 2, n_tokens, true);
@@ -381,7 +393,8 @@ modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const m
     }
     MODSE_STAGE(tm, 11, launch_router_bwd(dtype, m, x, weights->w_router, n_tokens, L.nblk_bwd, p, dx, of32,
                                           static_cast<float *>(wgrads->dw_router),
-                                          layer->aux_alpha * (float)m.N / (float)n_tokens, s, &launches));
+                                          layer->aux_alpha * (float)m.N / (float)n_tokens, layer->noise, s,
+                                          &launches));
     layer->last_launches = launches;
     return MODSE_OK;
 }
@@ -453,6 +466,24 @@ modse_status_t modse_aux_loss(modse_layer_t *layer, const void *workspace, int n
     MODSE_CUDA(launch_aux_loss(layer->meta, n_tokens, L.nblk_bwd, p, alpha, loss, f, P,
                                static_cast<cudaStream_t>(cuda_stream), &launches));
     layer->last_launches = launches;
+    return MODSE_OK;
+}
+
+modse_status_t modse_set_noise_gate(modse_layer_t *layer, const void *w_noise, float gamma, float eps)
+{
+    if (layer == nullptr || !(eps >= 0.f) || !(gamma == gamma)) return MODSE_ERR_INVALID_ARG;
+    if (w_noise != nullptr && !aligned16(w_noise)) return MODSE_ERR_INVALID_ARG;
+    layer->noise.w_noise = w_noise;
+    layer->noise.gamma = gamma;
+    layer->noise.eps = eps;
+    return MODSE_OK;
+}
+
+modse_status_t modse_set_noise_grads(modse_layer_t *layer, float *dw_noise, float *dgamma)
+{
+    if (layer == nullptr) return MODSE_ERR_INVALID_ARG;
+    layer->noise.dw_noise = dw_noise;
+    layer->noise.dgamma = dgamma;
     return MODSE_OK;
 }
 

@@ -31,7 +31,7 @@ struct WsLayout {
     int T, R, Pmax, nblk, nblk_bwd;
     size_t hb;   // element capacity of each [padded rows x h_e] activation buffer
     size_t status, topk_idx, topk_gate, counts, counts_slot, offsets, poffsets, ebase, row_of, token_of,
-        prow_of, ptoken_of, pgate, block_counts, logits, aux_partial, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
+        prow_of, ptoken_of, pgate, block_counts, logits, aux_partial, noise_u, du, dgamma_partial, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
         total;
 };
 
@@ -46,8 +46,20 @@ struct WsPtrs {
     int *block_counts;
     float *logits;       // [T,N] router logits (may be null: not stored)
     float *aux_partial;  // [nblk_bwd][N] partial sums of the router probabilities
+    float *noise_u;      // [T,N] x W_n, kept for the backward of the second term of Eq. 2
+    float *du;           // [T,N] gradient w.r.t. x W_n
+    float *dgamma_partial;  // [nblk_bwd]
     float *dg, *dz, *dwr_partial;
     void *xp, *a_pre, *b_pre, *hm, *o, *dyp, *da, *db, *dxp;
+};
+
+// Second term of the router logits (Sec. 2, Eq. 2): RMSNorm(Softplus(x W_n)) over the expert
+// entries, with scalar gamma.  w_noise == nullptr: the term is absent.
+struct NoiseGate {
+    const void *w_noise = nullptr;   // [N,d], layer dtype
+    float gamma = 0.f, eps = 0.f;
+    float *dw_noise = nullptr;       // [N,d] fp32
+    float *dgamma = nullptr;         // one float
 };
 
 WsLayout make_layout(const LayerMeta &m, const int *h_sorted_desc, int elem_bytes, int T, bool save);
@@ -55,7 +67,7 @@ WsPtrs carve(void *ws, const WsLayout &L);
 
 // ---- routing / permutation / elementwise stages (routing_kernels.cu) ----
 cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
-                          const WsPtrs &p, cudaStream_t s, int *launches);
+                          const WsPtrs &p, const NoiseGate &ng, cudaStream_t s, int *launches);
 cudaError_t launch_rank(const LayerMeta &m, int T, int Pmax, const WsPtrs &p, cudaStream_t s, int *launches);
 cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, const WsPtrs &p,
                            cudaStream_t s, int *launches);
@@ -66,7 +78,7 @@ cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *
 // aux_scale = alpha * N / T of the auxiliary load-balance loss (Eq. 7), 0 when it is not part of the objective
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
                               int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
-                              float aux_scale, cudaStream_t s, int *launches);
+                              float aux_scale, const NoiseGate &ng, cudaStream_t s, int *launches);
 // L_a = alpha N sum_i f_i P_i (Eq. 7-10) from the stored logits and the slot-0 histogram
 cudaError_t launch_aux_loss(const LayerMeta &m, int T, int nblk_bwd, const WsPtrs &p, float alpha, float *loss,
                             float *f, float *P, cudaStream_t s, int *launches);

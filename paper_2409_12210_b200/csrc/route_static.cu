@@ -108,7 +108,7 @@ extern "C" modse_status_t modse_route_static_scratch(modse_dtype_t dtype, int d_
     // the array keeps the previous call's bytes: the status word must start at zero, every
     // other region is fully rewritten by the two kernels before it is read
     if (cudaMemsetAsync(p.status, 0, 64, s) != cudaSuccess) return MODSE_ERR_CUDA;
-    if (launch_router(dtype, m, x, w_router, n_tokens, p, s, nullptr) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (launch_router(dtype, m, x, w_router, n_tokens, p, NoiseGate{}, s, nullptr) != cudaSuccess) return MODSE_ERR_CUDA;
     if (launch_rank(m, n_tokens, Pmax, p, s, nullptr) != cudaSuccess) return MODSE_ERR_CUDA;
     return MODSE_OK;
 }

@@ -72,56 +72,91 @@ constexpr int kNoIndex = 0x7FFFFFFF;
 // Router: one warp per token.  Each lane accumulates its 8-element chunks of
 // the row in ascending order with fp32 FMAs, then a butterfly adds the lanes.
 // ---------------------------------------------------------------------------
+// z[i] = <x_t, w[i]> for i < N, written by lane 0 (callers __syncwarp before reading)
+template <typename T>
+__device__ __forceinline__ void warp_row_dots(const T *__restrict__ xr, const T *__restrict__ w, int d, int N, int lane,
+                                              float *__restrict__ z)
+{
+    for (int g0 = 0; g0 < N; g0 += 8) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int c = lane * 8; c < d; c += 256) {
+            float xv[8];
+            load8(xr + c, xv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                if (g0 + i < N) {
+                    float wv[8];
+                    load8(w + (size_t)(g0 + i) * d + c, wv);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) acc[i] = fmaf(xv[u], wv[u], acc[i]);
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float s = warp_sum(acc[i]);
+            if (lane == 0 && g0 + i < N) z[g0 + i] = s;
+        }
+    }
+}
+
+// Softplus(u) = log(1 + exp(u)), written so that neither tail overflows or cancels.
+__device__ __forceinline__ float softplus_f(float u) { return u > 0.f ? u + log1pf(expf(-u)) : log1pf(expf(u)); }
+__device__ __forceinline__ float sigmoid_f(float u) { return 1.0f / (1.0f + expf(-u)); }
+
+// With w_noise != nullptr the logits carry the second term of Eq. 2,
+// H(x)_i = (x W_g)_i + gamma s_i / sqrt(mean_j s_j^2 + eps), s = Softplus(x W_n), and
+// noise_u [T,N] receives x W_n for the backward pass.
 template <typename T>
 __global__ void __launch_bounds__(256)
 router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok, int d, int N, int k,
               int *__restrict__ topk_idx, float *__restrict__ topk_gate, int *__restrict__ block_counts,
-              float *__restrict__ logits, int w_in_smem)
+              float *__restrict__ logits, int w_in_smem, const T *__restrict__ w_noise, float gamma, float eps,
+              float *__restrict__ noise_u)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int Npad = (N + 3) & ~3;
     int *cnt = reinterpret_cast<int *>(smem_raw);                                          // [k*N]
-    float *zbuf = reinterpret_cast<float *>(smem_raw + sizeof(int) * ((k * N + 3) & ~3));  // [8][Npad]
-    T *wsm = reinterpret_cast<T *>(reinterpret_cast<unsigned char *>(zbuf) + sizeof(float) * 8 * Npad);
+    float *zbuf = reinterpret_cast<float *>(smem_raw + sizeof(int) * ((k * N + 3) & ~3));  // [8][2][Npad]
+    T *wsm = reinterpret_cast<T *>(reinterpret_cast<unsigned char *>(zbuf) + sizeof(float) * 16 * Npad);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     for (int i = tid; i < k * N; i += blockDim.x) cnt[i] = 0;
-    const T *w = w_router;
+    const T *w = w_router, *wn = w_noise;
     if (w_in_smem) {
         const size_t bytes = (size_t)N * d * sizeof(T);   // a multiple of 16: d is a multiple of 8
-        const unsigned char *src = reinterpret_cast<const unsigned char *>(w_router);
         unsigned char *dst = reinterpret_cast<unsigned char *>(wsm);
-        for (size_t i = (size_t)tid * 16; i < bytes; i += (size_t)blockDim.x * 16)
-            *reinterpret_cast<uint4 *>(dst + i) = *reinterpret_cast<const uint4 *>(src + i);
+        for (int which = 0; which < (w_noise != nullptr ? 2 : 1); ++which) {
+            const unsigned char *src = reinterpret_cast<const unsigned char *>(which ? w_noise : w_router);
+            for (size_t i = (size_t)tid * 16; i < bytes; i += (size_t)blockDim.x * 16)
+                *reinterpret_cast<uint4 *>(dst + which * bytes + i) = *reinterpret_cast<const uint4 *>(src + i);
+        }
         w = wsm;
+        wn = wsm + (size_t)N * d;
     }
     __syncthreads();
 
-    float *z = zbuf + warp * Npad;
+    float *z = zbuf + warp * 2 * Npad;
+    float *un = z + Npad;
     const int t0 = blockIdx.x * kRouterTokB;
     for (int tok = warp; tok < kRouterTokB; tok += 8) {
         const int t = t0 + tok;
         if (t >= Ttok) break;
         const T *xr = x + (size_t)t * d;
-        for (int g0 = 0; g0 < N; g0 += 8) {
-            float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            for (int c = lane * 8; c < d; c += 256) {
-                float xv[8];
-                load8(xr + c, xv);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    if (g0 + i < N) {
-                        float wv[8];
-                        load8(w + (size_t)(g0 + i) * d + c, wv);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) acc[i] = fmaf(xv[u], wv[u], acc[i]);
-                    }
-                }
+        warp_row_dots(xr, w, d, N, lane, z);
+        if (w_noise != nullptr) {
+            warp_row_dots(xr, wn, d, N, lane, un);
+            __syncwarp();
+            float ss = 0.f;
+            for (int i = lane; i < N; i += 32) {
+                const float sp = softplus_f(un[i]);
+                ss = fmaf(sp, sp, ss);
             }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                float s = warp_sum(acc[i]);
-                if (lane == 0 && g0 + i < N) z[g0 + i] = s;
+            ss = warp_sum(ss);
+            const float scale = gamma / sqrtf(ss / (float)N + eps);
+            for (int i = lane; i < N; i += 32) {
+                noise_u[(size_t)t * N + i] = un[i];
+                z[i] = fmaf(softplus_f(un[i]), scale, z[i]);
             }
         }
         __syncwarp();
@@ -202,17 +237,21 @@ __device__ __forceinline__ void quad_argmax(float &bv, int &bi)
 constexpr int kRouterKSplit = 4;     // warps per 16-token group, each summing a quarter of the k range
 constexpr int kRouterMmaThreads = 4 * kRouterKSplit * 32;
 
-template <int NT>
+// NOISE: the rows of W_n are staged behind those of W_g and accumulated as NT more n-tiles, so a lane
+// holds (x W_g)_e and (x W_n)_e of the same experts e; the second term of Eq. 2 is added before top-k.
+template <int NT, bool NOISE>
 __global__ void __launch_bounds__(kRouterMmaThreads, 2)      // two 512-thread blocks per SM: at most 64 registers
 router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w_router, int Ttok, int d,
                   int N, int k, int *__restrict__ topk_idx, float *__restrict__ topk_gate,
-                  int *__restrict__ block_counts, float *__restrict__ logits)
+                  int *__restrict__ block_counts, float *__restrict__ logits,
+                  const __nv_bfloat16 *__restrict__ w_noise, float gamma, float eps, float *__restrict__ noise_u)
 {
+    constexpr int NTT = NOISE ? 2 * NT : NT;            // n-tiles accumulated per warp
     extern __shared__ __align__(16) unsigned char smem_raw[];
     int *cnt = reinterpret_cast<int *>(smem_raw);                                   // [k*N], padded to 128 bytes
-    float *part = reinterpret_cast<float *>(smem_raw + 128);                        // [KS-1][4 groups][32 lanes][NT*4]
+    float *part = reinterpret_cast<float *>(smem_raw + 128);                        // [KS-1][4 groups][32 lanes][NTT*4]
     __nv_bfloat16 *wsm = reinterpret_cast<__nv_bfloat16 *>(smem_raw + 128 +
-                                                           (kRouterKSplit - 1) * 4 * 32 * NT * 4 * sizeof(float));
+                                                           (kRouterKSplit - 1) * 4 * 32 * NTT * 4 * sizeof(float));
     const int ldw = d + 8;                                                          // 16-byte skew: conflict-free rows
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, tq = lane & 3;
@@ -236,24 +275,26 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
         xb[u] = (v1 && u < niter) ? x1[c0 >> 3] : za;
     }
     for (int i = tid; i < k * N; i += kRouterMmaThreads) cnt[i] = 0;
-    for (int i = tid * 8; i < NT * 8 * d; i += kRouterMmaThreads * 8) {
+    for (int i = tid * 8; i < NTT * 8 * d; i += kRouterMmaThreads * 8) {
         const int r = i / d, c = i % d;
+        const int e = r < NT * 8 ? r : r - NT * 8;          // rows [NT*8, 2*NT*8) hold W_n
+        const __nv_bfloat16 *src = r < NT * 8 ? w_router : w_noise;
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (r < N) v = *reinterpret_cast<const uint4 *>(w_router + (size_t)r * d + c);
+        if (e < N) v = *reinterpret_cast<const uint4 *>(src + (size_t)e * d + c);
         *reinterpret_cast<uint4 *>(wsm + (size_t)r * ldw + c) = v;
     }
     __syncthreads();
 
-    float acc[NT][4];
+    float acc[NTT][4];
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+    for (int nt = 0; nt < NTT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
     for (int it0 = 0; it0 < niter; it0 += UB) {
 #pragma unroll
         for (int u = 0; u < UB; ++u) {
             const int c0 = cbeg + (it0 + u) * 32;
             if (it0 + u < niter) {
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
+                for (int nt = 0; nt < NTT; ++nt) {
                     const uint4 w = *reinterpret_cast<const uint4 *>(wsm + (size_t)(nt * 8 + g) * ldw + c0 + tq * 8);
                     mma_bf16_16816(acc[nt], xa[u].x, xb[u].x, xa[u].y, xb[u].y, w.x, w.y);
                     mma_bf16_16816(acc[nt], xa[u].z, xb[u].z, xa[u].w, xb[u].w, w.z, w.w);
@@ -270,21 +311,46 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
     // which adds them in a fixed order
     if (kpart > 0) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int nt = 0; nt < NTT; ++nt)
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                part[((((kpart - 1) * 4 + grp) * 32 + lane) * NT + nt) * 4 + u] = acc[nt][u];
+                part[((((kpart - 1) * 4 + grp) * 32 + lane) * NTT + nt) * 4 + u] = acc[nt][u];
     }
     __syncthreads();
     if (kpart == 0) {
 #pragma unroll
         for (int q = 1; q < kRouterKSplit; ++q)
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
+            for (int nt = 0; nt < NTT; ++nt)
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    acc[nt][u] += part[((((q - 1) * 4 + grp) * 32 + lane) * NT + nt) * 4 + u];
+                    acc[nt][u] += part[((((q - 1) * 4 + grp) * 32 + lane) * NTT + nt) * 4 + u];
         // acc[nt][0..1]: token r0, experts nt*8 + 2tq, +1;  acc[nt][2..3]: token r1, same experts
+        if constexpr (NOISE) {
+            // acc[NT + nt] holds x W_n of the same experts: add gamma s / sqrt(mean s^2 + eps), s = Softplus
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                const int t = half ? r1 : r0;
+                float sp[NT][2], ss = 0.f;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int e = nt * 8 + 2 * tq + u;
+                        const float un = acc[NT + nt][2 * half + u];
+                        sp[nt][u] = e < N ? softplus_f(un) : 0.f;
+                        ss = fmaf(sp[nt][u], sp[nt][u], ss);
+                        if (t < Ttok && e < N) noise_u[(size_t)t * N + e] = un;
+                    }
+                ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 1);
+                ss += __shfl_xor_sync(0xFFFFFFFFu, ss, 2);
+                const float scale = gamma / sqrtf(ss / (float)N + eps);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) acc[nt][2 * half + u] = fmaf(sp[nt][u], scale, acc[nt][2 * half + u]);
+            }
+        }
         if (logits != nullptr) {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
@@ -634,8 +700,87 @@ aux_final_kernel(const float *__restrict__ partial, int nblk, const int *__restr
 }
 
 // ---------------------------------------------------------------------------
+// Backward of the second term of Eq. 2 (thread per token).  With dz = dL/dH over all N
+// entries of the token (softmax Jacobian on the kept logits plus the auxiliary-loss term),
+// s = Softplus(u), q = sqrt(mean s^2 + eps):
+//   dgamma_t = sum_i dz_i s_i / q
+//   du_i = gamma (dz_i / q - s_i (sum_j dz_j s_j) / (N q^3)) sigmoid(u_i)
+// du [T,N] feeds dW_n = du^T x and dx += du W_n; dgamma_t is summed over the block's tokens
+// in token order (block order in reduce_scalar_kernel).
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(kRouterBwdTokB)
+noise_bwd_kernel(const float *__restrict__ noise_u, int Ttok, int N, int k, const int *__restrict__ topk_idx,
+                 const float *__restrict__ topk_gate, const float *__restrict__ dg,
+                 const float *__restrict__ logits, const int *__restrict__ counts_slot, float aux_scale,
+                 float gamma, float eps, float *__restrict__ du, float *__restrict__ dgamma_partial)
+{
+    __shared__ float dgt[kRouterBwdTokB];
+    const int tid = threadIdx.x;
+    const int t = blockIdx.x * kRouterBwdTokB + tid;
+    float dgamma_t = 0.f;
+    if (t < Ttok) {
+        int e[2] = {-1, -1};
+        float dzk[2] = {0.f, 0.f};
+        {
+            float g[2] = {0.f, 0.f}, dgv[2] = {0.f, 0.f};
+            for (int j = 0; j < k; ++j) {
+                g[j] = topk_gate[(size_t)t * k + j];
+                dgv[j] = dg[(size_t)t * k + j];
+                e[j] = topk_idx[(size_t)t * k + j];
+            }
+            const float sg = g[0] * dgv[0] + g[1] * dgv[1];
+            dzk[0] = g[0] * (dgv[0] - sg);
+            dzk[1] = g[1] * (dgv[1] - sg);
+        }
+        const float *u = noise_u + (size_t)t * N;
+        const float *zt = logits + (size_t)t * N;
+        const float inv_T = 1.0f / (float)Ttok;
+        float zmax = 0.f, inv_den = 0.f, fp = 0.f;
+        if (aux_scale != 0.f) token_softmax_stats(zt, counts_slot, N, inv_T, zmax, inv_den, fp);
+        auto dz_at = [&](int i) {
+            float v = 0.f;
+            if (i == e[0]) v = dzk[0];
+            if (i == e[1]) v = dzk[1];
+            if (aux_scale != 0.f)
+                v += aux_scale * expf(zt[i] - zmax) * inv_den * ((float)counts_slot[i] * inv_T - fp);
+            return v;
+        };
+        float ms = 0.f, dzs = 0.f;
+        for (int i = 0; i < N; ++i) {
+            const float sp = softplus_f(u[i]);
+            ms = fmaf(sp, sp, ms);
+            dzs = fmaf(dz_at(i), sp, dzs);
+        }
+        const float q = sqrtf(ms / (float)N + eps);
+        dgamma_t = dzs / q;
+        const float c1 = gamma / q, c2 = gamma * dzs / ((float)N * q * q * q);
+        for (int i = 0; i < N; ++i) {
+            const float sp = softplus_f(u[i]);
+            du[(size_t)t * N + i] = (c1 * dz_at(i) - c2 * sp) * sigmoid_f(u[i]);
+        }
+    }
+    dgt[tid] = dgamma_t;
+    __syncthreads();
+    if (tid == 0) {
+        float acc = 0.f;
+        for (int i = 0; i < kRouterBwdTokB; ++i) acc += dgt[i];
+        dgamma_partial[blockIdx.x] = acc;
+    }
+}
+
+__global__ void reduce_scalar_kernel(const float *__restrict__ partial, int n, float *__restrict__ out)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        float acc = 0.f;
+        for (int i = 0; i < n; ++i) acc += partial[i];
+        *out = acc;
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Router backward, part 1 (warp per token): s = sum_j g_j dg_j,
-// dz_j = g_j (dg_j - s), dx_t = sum_j dxp[row_j] + sum_j dz_j W_router[e_j].
+// dz_j = g_j (dg_j - s), dx_t = sum_j dxp[row_j] + sum_j dz_j W_router[e_j]
+// (+ sum_m du_m W_n[m] when the logits carry the second term of Eq. 2).
 // ---------------------------------------------------------------------------
 template <typename T, typename TO>
 __global__ void __launch_bounds__(256)
@@ -643,7 +788,7 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
                  const int *__restrict__ topk_idx, const float *__restrict__ topk_gate,
                  const int *__restrict__ prow_of, const float *__restrict__ dg, float *__restrict__ dz,
                  TO *__restrict__ dx, int N, const float *__restrict__ logits, const int *__restrict__ counts_slot,
-                 float aux_scale)
+                 float aux_scale, const T *__restrict__ w_noise, const float *__restrict__ du)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * 8 + warp;
@@ -687,6 +832,14 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
                 for (int u = 0; u < 8; ++u) out[u] = fmaf(dza, wv[u], out[u]);
             }
         }
+        if (w_noise != nullptr) {
+            for (int m = 0; m < N; ++m) {
+                const float dum = du[(size_t)t * N + m];
+                load8(w_noise + (size_t)m * d + c, wv);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) out[u] = fmaf(dum, wv[u], out[u]);
+            }
+        }
         store8(dx + (size_t)t * d + c, out);
     }
 }
@@ -695,13 +848,14 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
 // Router backward, part 2: dW_router = dz^T x as per-block partial sums.  Block
 // (bx, by) owns tokens [128 bx, +128) and columns [256 by, +256); each thread
 // owns one column and adds its tokens in ascending order, eight experts at a
-// time, against the dense [128][8] slice of dz held in shared memory.
+// time, against the dense [128][8] slice of dz held in shared memory.  With `dense`
+// set, the slice is read from that [T,N] array instead (dW_n = du^T x).
 // ---------------------------------------------------------------------------
 template <typename T>
 __global__ void __launch_bounds__(256)
 router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int *__restrict__ topk_idx,
                   const float *__restrict__ dz, float *__restrict__ dwr_partial, const float *__restrict__ logits,
-                  const int *__restrict__ counts_slot, float aux_scale)
+                  const int *__restrict__ counts_slot, float aux_scale, const float *__restrict__ dense)
 {
     constexpr int CPT = (sizeof(T) == 2) ? 2 : 1;        // columns per thread: one 4-byte load either way
     __shared__ float dzs[kRouterBwdTokB][8];
@@ -726,9 +880,13 @@ router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const 
         for (int i = tid; i < kRouterBwdTokB * 8; i += 256) {
             const int tl = i >> 3, e = g0 + (i & 7);
             float v = 0.f;
-            if (idxs[tl][0] == e) v = dzk[tl][0];
-            if (idxs[tl][1] == e) v = dzk[tl][1];
-            if (aux_scale != 0.f && tl < ntok && e < N) {
+            if (dense != nullptr) {
+                if (tl < ntok && e < N) v = dense[(size_t)(t0 + tl) * N + e];
+            } else {
+                if (idxs[tl][0] == e) v = dzk[tl][0];
+                if (idxs[tl][1] == e) v = dzk[tl][1];
+            }
+            if (dense == nullptr && aux_scale != 0.f && tl < ntok && e < N) {
                 const float pm = expf(logits[(size_t)(t0 + tl) * N + e] - smax[tl]) * sinv[tl];
                 v += aux_scale * pm * ((float)counts_slot[e] * inv_T - sfp[tl]);
             }
@@ -790,26 +948,29 @@ reduce_dwr_kernel(const float *__restrict__ partial, int nblk, int n, float *__r
     } while (0)
 
 cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
-                          const WsPtrs &p, cudaStream_t s, int *launches)
+                          const WsPtrs &p, const NoiseGate &ng, cudaStream_t s, int *launches)
 {
     const int nblk = (T + kRouterTokB - 1) / kRouterTokB;
+    const bool noise = ng.w_noise != nullptr;
     if (dt == MODSE_BF16 && m.N <= 16 && m.d % (32 * kRouterKSplit) == 0 && m.k * m.N * 4 <= 128) {
-        const int nt = (m.N + 7) / 8;
-        const size_t smem = 128 + (size_t)(kRouterKSplit - 1) * 4 * 32 * nt * 4 * sizeof(float) +
-                            (size_t)nt * 8 * (m.d + 8) * 2;
-        if (smem <= 200 * 1024) {
-            auto kern = nt == 1 ? router_mma_kernel<1> : router_mma_kernel<2>;
+        const int nt = (m.N + 7) / 8, ntt = noise ? 2 * nt : nt;
+        const size_t smem = 128 + (size_t)(kRouterKSplit - 1) * 4 * 32 * ntt * 4 * sizeof(float) +
+                            (size_t)ntt * 8 * (m.d + 8) * 2;
+        if (smem <= 200 * 1024 && !(noise && nt > 1)) {
+            auto kern = noise ? router_mma_kernel<1, true>
+                              : (nt == 1 ? router_mma_kernel<1, false> : router_mma_kernel<2, false>);
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
             kern<<<nblk, kRouterMmaThreads, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
-                                         p.topk_idx, p.topk_gate, p.block_counts, p.logits);
+                                         p.topk_idx, p.topk_gate, p.block_counts, p.logits,
+                                         (const __nv_bfloat16 *)ng.w_noise, ng.gamma, ng.eps, p.noise_u);
             MODSE_LAUNCH_CHECK();
             return cudaSuccess;
         }
     }
     const size_t esz = dt == MODSE_F32 ? 4 : 2;
-    const size_t base = sizeof(int) * ((m.k * m.N + 3) & ~3) + sizeof(float) * 8 * ((m.N + 3) & ~3);
-    const size_t wbytes = (size_t)m.N * m.d * esz;
+    const size_t base = sizeof(int) * ((m.k * m.N + 3) & ~3) + sizeof(float) * 16 * ((m.N + 3) & ~3);
+    const size_t wbytes = (size_t)m.N * m.d * esz * (noise ? 2 : 1);
     const int w_in_smem = (base + wbytes <= 160 * 1024) ? 1 : 0;
     const size_t smem = base + (w_in_smem ? wbytes : 0);
     if (dt == MODSE_F32) {
@@ -817,13 +978,15 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<nblk, 256, smem, s>>>((const float *)x, (const float *)w_router, T, m.d, m.N, m.k, p.topk_idx,
-                                     p.topk_gate, p.block_counts, p.logits, w_in_smem);
+                                     p.topk_gate, p.block_counts, p.logits, w_in_smem, (const float *)ng.w_noise,
+                                     ng.gamma, ng.eps, p.noise_u);
     } else {
         auto kern = router_kernel<__nv_bfloat16>;
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<nblk, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
-                                     p.topk_idx, p.topk_gate, p.block_counts, p.logits, w_in_smem);
+                                     p.topk_idx, p.topk_gate, p.block_counts, p.logits, w_in_smem,
+                                     (const __nv_bfloat16 *)ng.w_noise, ng.gamma, ng.eps, p.noise_u);
     }
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
@@ -889,35 +1052,51 @@ cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *
 
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
                               int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
-                              float aux_scale, cudaStream_t s, int *launches)
+                              float aux_scale, const NoiseGate &ng, cudaStream_t s, int *launches)
 {
+    const bool noise = ng.w_noise != nullptr;
+    const float *du = noise ? p.du : nullptr;
+    if (noise) {
+        noise_bwd_kernel<<<nblk_bwd, kRouterBwdTokB, 0, s>>>(p.noise_u, T, m.N, m.k, p.topk_idx, p.topk_gate, p.dg,
+                                                             p.logits, p.counts_slot, aux_scale, ng.gamma, ng.eps,
+                                                             p.du, p.dgamma_partial);
+        MODSE_LAUNCH_CHECK();
+        reduce_scalar_kernel<<<1, 32, 0, s>>>(p.dgamma_partial, nblk_bwd, ng.dgamma);
+        MODSE_LAUNCH_CHECK();
+    }
     const int grid_dx = (T + 7) / 8;
     const float *dxp = (const float *)p.dxp;
     if (dt == MODSE_F32)
         router_dx_kernel<float, float><<<grid_dx, 256, 0, s>>>((const float *)w_router, dxp, T, m.d, m.k, p.topk_idx,
                                                                p.topk_gate, p.prow_of, p.dg, p.dz, (float *)dx, m.N, p.logits,
-                                                               p.counts_slot, aux_scale);
+                                                               p.counts_slot, aux_scale, (const float *)ng.w_noise, du);
     else if (out_f32)
         router_dx_kernel<__nv_bfloat16, float><<<grid_dx, 256, 0, s>>>((const __nv_bfloat16 *)w_router, dxp, T, m.d,
                                                                        m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg,
                                                                        p.dz, (float *)dx, m.N, p.logits, p.counts_slot,
-                                                                       aux_scale);
+                                                                       aux_scale, (const __nv_bfloat16 *)ng.w_noise, du);
     else
         router_dx_kernel<__nv_bfloat16, __nv_bfloat16><<<grid_dx, 256, 0, s>>>(
             (const __nv_bfloat16 *)w_router, dxp, T, m.d, m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz,
-            (__nv_bfloat16 *)dx, m.N, p.logits, p.counts_slot, aux_scale);
+            (__nv_bfloat16 *)dx, m.N, p.logits, p.counts_slot, aux_scale, (const __nv_bfloat16 *)ng.w_noise, du);
     MODSE_LAUNCH_CHECK();
     dim3 grid(nblk_bwd, dt == MODSE_F32 ? (m.d + 255) / 256 : (m.d + 511) / 512);
-    if (dt == MODSE_F32)
-        router_dwr_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.topk_idx, p.dz,
-                                                      p.dwr_partial, p.logits, p.counts_slot, aux_scale);
-    else
-        router_dwr_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k, p.topk_idx,
-                                                              p.dz, p.dwr_partial, p.logits, p.counts_slot, aux_scale);
-    MODSE_LAUNCH_CHECK();
     const int n = m.N * m.d;
-    reduce_dwr_kernel<<<(n + 255) / 256, 256, 0, s>>>(p.dwr_partial, nblk_bwd, n, dw_router);
-    MODSE_LAUNCH_CHECK();
+    // pass 0: dW_router = dz^T x;  pass 1 (second term only): dW_n = du^T x through the same partial buffer
+    for (int pass = 0; pass < (noise ? 2 : 1); ++pass) {
+        const float *dense = pass ? du : nullptr;
+        const float ascale = pass ? 0.f : aux_scale;
+        if (dt == MODSE_F32)
+            router_dwr_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.topk_idx, p.dz,
+                                                          p.dwr_partial, p.logits, p.counts_slot, ascale, dense);
+        else
+            router_dwr_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k,
+                                                                  p.topk_idx, p.dz, p.dwr_partial, p.logits,
+                                                                  p.counts_slot, ascale, dense);
+        MODSE_LAUNCH_CHECK();
+        reduce_dwr_kernel<<<(n + 255) / 256, 256, 0, s>>>(p.dwr_partial, nblk_bwd, n, pass ? ng.dw_noise : dw_router);
+        MODSE_LAUNCH_CHECK();
+    }
     return cudaSuccess;
 }
 

@@ -87,3 +87,18 @@ def test_forward_argument_errors_need_no_gpu():
                             0x1000, n, None)
     assert st == B.MODSE_ERR_STATE                                 # no forward was saved
     layer.destroy()
+
+
+def test_noise_gate_argument_errors_need_no_gpu():
+    lib = B.load()
+    layer = B.ModseLayer(64, [96, 160, 112, 144], 2)
+    cf = ctypes.c_float
+    assert lib.modse_set_noise_gate(None, 0x1000, cf(1.0), cf(1e-6)) == B.MODSE_ERR_INVALID_ARG
+    assert lib.modse_set_noise_gate(layer._h, 0x1004, cf(1.0), cf(1e-6)) == B.MODSE_ERR_INVALID_ARG   # alignment
+    assert lib.modse_set_noise_gate(layer._h, 0x1000, cf(1.0), cf(-1.0)) == B.MODSE_ERR_INVALID_ARG   # eps < 0
+    assert lib.modse_set_noise_gate(layer._h, 0x1000, cf(float("nan")), cf(0.0)) == B.MODSE_ERR_INVALID_ARG
+    assert lib.modse_set_noise_gate(layer._h, 0x1000, cf(1.0), cf(1e-6)) == B.MODSE_OK
+    assert lib.modse_set_noise_gate(layer._h, None, cf(0.0), cf(0.0)) == B.MODSE_OK                   # off again
+    assert lib.modse_set_noise_grads(None, 0x1000, 0x1000) == B.MODSE_ERR_INVALID_ARG
+    assert lib.modse_set_noise_grads(layer._h, 0x1000, 0x1000) == B.MODSE_OK
+    layer.destroy()
