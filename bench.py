@@ -219,6 +219,11 @@ def main():
     ap.add_argument("--tokens", type=int, default=None, help="override the workload's token count")
     ap.add_argument("--layers", type=int, default=1,
                     help="layer-stack sweep: a step runs this many independent layers (own weights, x and dY each)")
+    ap.add_argument("--noise-gate", action="store_true",
+                    help="add the second router term RMSNorm(Softplus(x W_n)) (Eq. 2) to the logits; off in the "
+                         "default benchmark, whose router is x W_g alone")
+    ap.add_argument("--aux-alpha", type=float, default=0.0,
+                    help="coefficient of the auxiliary load-balance loss (Eq. 7) added to the objective in backward")
     ap.add_argument("--pair-mask", type=int, default=None,
                     help="tuning: which grouped products use the two-SM kernel (bit per product)")
     args = ap.parse_args()
@@ -266,6 +271,15 @@ def main():
     dwr = torch.empty(wr.shape, dtype=torch.float32, device=dev)
     dwg, dwu, dwd = torch.empty_like(wg), torch.empty_like(wu), torch.empty_like(wd)
     do_bwd = cfg.backward
+    if args.noise_gate:
+        gen = torch.Generator(device=dev).manual_seed(cfg.seed + 4242)
+        w_noise = (torch.randn(wr.shape, generator=gen, device=dev, dtype=torch.float32) * d ** -0.5).to(dt)
+        dw_noise = torch.empty(wr.shape, dtype=torch.float32, device=dev)
+        dgamma = torch.empty(1, dtype=torch.float32, device=dev)
+        layer.set_noise_gate(w_noise, 1.0, 1e-6)
+        layer.set_noise_grads(dw_noise, dgamma)
+    if args.aux_alpha > 0:
+        layer.set_aux_loss(args.aux_alpha)
     ws = layer.alloc_workspace(dt, T, do_bwd, dev)
 
     def step(xb=None, dyb=None, yb=None, dxb=None):
@@ -412,7 +426,7 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "d_model": d, "ffn_sizes": list(cfg.ffn_sizes), "top_k": cfg.top_k,
-                   "n_tokens": T, "layers": L,
+                   "n_tokens": T, "layers": L, "noise_gate": bool(args.noise_gate), "aux_alpha": args.aux_alpha,
                    "e2e_copies": "x, dY in and y, dx out of layer 0" if L > 1 else "x, dY in; y, dx out", "pass": "fwd+bwd" if do_bwd else "fwd", "parallelism": f"replicas x{world}",
                    "l2": "inputs larger than L2 (weights 554 MB, activations > 126 MB per step)"},
         "tflops": flops_step / (ms_step * 1e-3) / 1e12,

@@ -1,5 +1,5 @@
 """GPU parity at the full benchmark sizes (width 2048, 8 experts of diverse widths, top-2;
-8192 tokens forward-only and 16384 tokens forward+backward), in the launch configuration
+8192 tokens forward-only, 16384 and 65536 tokens forward+backward), in the launch configuration
 bench.py times.  The routing tables are compared in full (bit-exact); floating outputs are
 compared on sampled tokens / sampled weight-gradient rows that the fp64 oracle computes one
 by one, and dW_router through the identity dW_router = dz^T x."""
@@ -73,7 +73,7 @@ def compare(gpu, ora, cfg, backward, discount):
     return errs
 
 
-@pytest.mark.parametrize("name", ["fwd_8k", "train_16k", "train_16k_skew", "table2_700m", "table2_300m"])
+@pytest.mark.parametrize("name", ["fwd_8k", "train_16k", "train_16k_skew", "table2_700m", "table2_300m", "train_64k"])
 def test_full_size_sampled_parity(name):
     cfg = I.CONFIGS[name]
     inp, n_redrawn = H.screened(cfg)
