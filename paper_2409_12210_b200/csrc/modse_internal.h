@@ -50,6 +50,10 @@ struct WsPtrs {
     float *du;           // [T,N] gradient w.r.t. x W_n
     float *dgamma_partial;  // [nblk_bwd]
     float *dg, *dz, *dwr_partial;
+    // xp: x in padded expert-grouped rows.  a_pre / b_pre: what the forward keeps for the SwiGLU backward -
+    // the pre-activations A = xp W_gate^T, B = xp W_up^T on the fp32 path, B silu'(A) and silu(A) on the bf16
+    // path.  hm: gated hidden rows g silu(A) B.  o / dxp: fp32 gated expert outputs / input gradients per row.
+    // dyp: dY in group order.  da / db: gradients w.r.t. A and B.
     void *xp, *a_pre, *b_pre, *hm, *o, *dyp, *da, *db, *dxp;
 };
 
