@@ -177,6 +177,23 @@ modse_status_t modse_set_aux_loss(modse_layer_t *layer, float alpha);
  * accumulation over micro-batches in fp32.  No effect on fp32 layers.        */
 modse_status_t modse_set_output_f32(modse_layer_t *layer, int on);
 
+/* Choice of kernel shape per device (no counterpart in the paper: a property of this implementation).
+ * Each grouped product of the bf16 layer exists with 128-row and with 256-row tiles; which is faster for the
+ * two forward products depends on how fast the GPU at hand feeds shared memory from L2, which differs between
+ * otherwise identical boards.  modse_tune_forward runs the forward pass (arguments as modse_forward) a few
+ * times per candidate on the caller's own buffers, times it with CUDA events, and keeps the fastest plan in
+ * the layer object for all later calls.  It allocates no device memory, SYNCHRONISES the stream, and leaves y
+ * and the workspace as one modse_forward would.  Results do not depend on the plan (the K order of every sum
+ * is the same).  fp32 layers have one kernel shape: the call returns MODSE_OK at once.
+ * modse_get_tile_plan returns the plan (-1: library default; else bit k: product k on the two-SM kernel,
+ * bit 8+k: product k on the 256-row kernel, k = 0 up/gate, 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate
+ * dgrad, 5 up/gate wgrad); modse_set_tile_plan installs one (e.g. a plan found earlier on the same device). */
+modse_status_t modse_tune_forward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
+                                  const void *x, int n_tokens, void *y, void *workspace, size_t workspace_bytes,
+                                  int save_for_backward, void *cuda_stream);
+int modse_get_tile_plan(const modse_layer_t *layer);
+modse_status_t modse_set_tile_plan(modse_layer_t *layer, int plan);
+
 /* Second term of the router logits (Sec. 2, Eq. 2 with the RMSNorm and Softplus
  * definitions that follow it):
  *   H(x)_i = (x W_g)_i + RMSNorm(Softplus((x W_n)_i)),

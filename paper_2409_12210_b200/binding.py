@@ -95,6 +95,12 @@ def load():
     lib.modse_set_noise_gate.argtypes = [vp, vp, ctypes.c_float, ctypes.c_float]
     lib.modse_set_noise_grads.restype = ci
     lib.modse_set_noise_grads.argtypes = [vp, vp, vp]
+    lib.modse_tune_forward.restype = ci
+    lib.modse_tune_forward.argtypes = [vp, ci, ctypes.POINTER(_Weights), vp, ci, vp, vp, sz, ci, vp]
+    lib.modse_get_tile_plan.restype = ci
+    lib.modse_get_tile_plan.argtypes = [vp]
+    lib.modse_set_tile_plan.restype = ci
+    lib.modse_set_tile_plan.argtypes = [vp, ci]
     lib.modse_set_output_f32.restype = ci
     lib.modse_set_output_f32.argtypes = [vp, ci]
     lib.modse_stage_timing_begin.restype = ci
@@ -216,6 +222,25 @@ class ModseLayer:
                                   workspace.data_ptr(), workspace.numel(), int(save_for_backward), self._stream())
         if st != MODSE_OK:
             raise ModseError(st, "modse_forward")
+
+    def tune_forward(self, w_router, w_gate, w_up, w_down, x, y, workspace, save_for_backward: bool) -> int:
+        """Time the kernel shapes of the forward products on this device (synchronises) and keep the fastest;
+        returns the plan (see modse_get_tile_plan)."""
+        w = _Weights(w_router.data_ptr(), w_gate.data_ptr(), w_up.data_ptr(), w_down.data_ptr())
+        st = load().modse_tune_forward(self._h, _dtype_code(x), ctypes.byref(w), x.data_ptr(), x.shape[0],
+                                       y.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                       int(save_for_backward), self._stream())
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_tune_forward")
+        return self.tile_plan()
+
+    def tile_plan(self) -> int:
+        return int(load().modse_get_tile_plan(self._h))
+
+    def set_tile_plan(self, plan: int) -> None:
+        st = load().modse_set_tile_plan(self._h, int(plan))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_set_tile_plan")
 
     def backward(self, w_router, w_gate, w_up, w_down, x, dy, dx, dw_router, dw_gate, dw_up, dw_down, workspace):
         w = _Weights(w_router.data_ptr(), w_gate.data_ptr(), w_up.data_ptr(), w_down.data_ptr())

@@ -487,6 +487,74 @@ modse_status_t modse_set_noise_grads(modse_layer_t *layer, float *dw_noise, floa
     return MODSE_OK;
 }
 
+modse_status_t modse_tune_forward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
+                                  const void *x, int n_tokens, void *y, void *workspace, size_t workspace_bytes,
+                                  int save_for_backward, void *cuda_stream)
+{
+    modse_status_t st = check_common(layer, dtype, weights, n_tokens, workspace, workspace_bytes, save_for_backward);
+    if (st != MODSE_OK) return st;
+    if (dtype != MODSE_BF16 || tc_force_simt() || n_tokens == 0) return MODSE_OK;   // one kernel shape only
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaEvent_t ev[2];
+    if (cudaEventCreate(&ev[0]) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (cudaEventCreate(&ev[1]) != cudaSuccess) { cudaEventDestroy(ev[0]); return MODSE_ERR_CUDA; }
+    const int prev = layer->tc.tile_mask;
+    const int base = prev >= 0 ? prev : tc_pair_mask();
+    const int fwd_bits = ((1 << TcUpGate) | (1 << TcDown)) * 0x101;      // both variant bits of the two forward products
+    // candidates: each forward product on the 128-row or on the 256-row kernel.  They are timed in
+    // interleaved rounds after a warm-up, so that the drift of the clocks under the power limit (a burst
+    // after idle, lower clocks later) does not favour whichever candidate runs first.
+    int masks[4];
+    float total_ms[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int cand = 0; cand < 4; ++cand) {
+        const int wide = ((cand & 1) ? (1 << TcUpGate) : 0) | ((cand & 2) ? (1 << TcDown) : 0);
+        masks[cand] = (base & ~fwd_bits) | (wide << 8);
+    }
+    auto run = [&](int reps) {
+        for (int rep = 0; rep < reps && st == MODSE_OK; ++rep)
+            st = modse_forward(layer, dtype, weights, x, n_tokens, y, workspace, workspace_bytes, save_for_backward,
+                               cuda_stream);
+    };
+    for (int cand = 0; cand < 4; ++cand) {          // warm-up: every candidate twice
+        layer->tc.tile_mask = masks[cand];
+        run(2);
+    }
+    for (int round = 0; round < 3 && st == MODSE_OK; ++round)
+        for (int cand = 0; cand < 4 && st == MODSE_OK; ++cand) {
+            layer->tc.tile_mask = masks[cand];
+            float ms = 0.f;
+            if (cudaEventRecord(ev[0], s) != cudaSuccess) st = MODSE_ERR_CUDA;
+            run(2);
+            if (st == MODSE_OK && (cudaEventRecord(ev[1], s) != cudaSuccess || cudaEventSynchronize(ev[1]) != cudaSuccess ||
+                                   cudaEventElapsedTime(&ms, ev[0], ev[1]) != cudaSuccess))
+                st = MODSE_ERR_CUDA;
+            total_ms[cand] += ms;
+        }
+    int best_mask = base;
+    if (st == MODSE_OK) {
+        int best = 0;
+        for (int cand = 1; cand < 4; ++cand)
+            if (total_ms[cand] < total_ms[best]) best = cand;
+        best_mask = masks[best];
+    }
+    cudaEventDestroy(ev[0]);
+    cudaEventDestroy(ev[1]);
+    layer->tc.tile_mask = st == MODSE_OK ? best_mask : prev;
+    if (st == MODSE_OK)      // leave y and the workspace as one forward under the chosen plan produces them
+        st = modse_forward(layer, dtype, weights, x, n_tokens, y, workspace, workspace_bytes, save_for_backward,
+                           cuda_stream);
+    return st;
+}
+
+int modse_get_tile_plan(const modse_layer_t *layer) { return layer ? layer->tc.tile_mask : -1; }
+
+modse_status_t modse_set_tile_plan(modse_layer_t *layer, int plan)
+{
+    if (layer == nullptr || (plan != -1 && (plan < 0 || (plan & ~0x3F3F) != 0))) return MODSE_ERR_INVALID_ARG;
+    layer->tc.tile_mask = plan;
+    return MODSE_OK;
+}
+
 modse_status_t modse_set_output_f32(modse_layer_t *layer, int on)
 {
     if (layer == nullptr) return MODSE_ERR_INVALID_ARG;

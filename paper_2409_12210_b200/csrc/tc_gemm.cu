@@ -443,7 +443,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     const float av = __uint_as_float(ra[i]), bv = __uint_as_float(rb[i]);
-                    const float sg = 1.0f / (1.0f + __expf(-av));
+                    const float sg = __fdividef(1.0f, 1.0f + __expf(-av));   // ex2 + rcp: a full-precision division here slows the MMA warp
                     sq[i] = av * sg;
                     sp[i] = bv * sg * (1.0f + av * (1.0f - sg));
                     hm[i] = gate * (sq[i] * bv);
@@ -454,7 +454,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
                     const float av = __uint_as_float(ra[i]), bv = __uint_as_float(rb[i]);
-                    hm[i] = gate * (av * (1.0f / (1.0f + __expf(-av))) * bv);
+                    hm[i] = gate * (av * __fdividef(1.0f, 1.0f + __expf(-av)) * bv);
                 }
             }
             store_bf16x32_staged(stg, lane, prm.hm + idx, 64, hm);
@@ -1528,10 +1528,10 @@ cudaError_t launch_kind_wide(const TcMaps &maps, const TcParams &prm, int grid, 
 }
 
 template <int KIND>
-cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
+cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, int mask, cudaStream_t s, int *launches)
 {
-    if (g_wide_mask & (1 << KIND)) return launch_kind_wide<KIND>(maps, prm, grid, s, launches);
-    if (g_pair_mask & (1 << KIND)) return launch_kind_pair<KIND>(maps, prm, grid, s, launches);
+    if ((mask >> 8) & (1 << KIND)) return launch_kind_wide<KIND>(maps, prm, grid, s, launches);
+    if (mask & (1 << KIND)) return launch_kind_pair<KIND>(maps, prm, grid, s, launches);
     auto kern = tc_grouped_gemm<KIND>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (e != cudaSuccess) return e;
@@ -1561,13 +1561,14 @@ cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const Layer
 {
     const TcParams prm = make_params(m, p, g, save, out_f32);
     const int grid = sm_count(plan);
+    const int mask = plan.tile_mask >= 0 ? plan.tile_mask : tc_pair_mask();
     switch (kind) {
-    case TcUpGate: return launch_kind<TcUpGate>(maps, prm, grid, s, launches);
-    case TcDown: return launch_kind<TcDown>(maps, prm, grid, s, launches);
-    case TcDownDgrad: return launch_kind<TcDownDgrad>(maps, prm, grid, s, launches);
-    case TcDownWgrad: return launch_kind<TcDownWgrad>(maps, prm, grid, s, launches);
-    case TcUpGateDgrad: return launch_kind<TcUpGateDgrad>(maps, prm, grid, s, launches);
-    case TcUpGateWgrad: return launch_kind<TcUpGateWgrad>(maps, prm, grid, s, launches);
+    case TcUpGate: return launch_kind<TcUpGate>(maps, prm, grid, mask, s, launches);
+    case TcDown: return launch_kind<TcDown>(maps, prm, grid, mask, s, launches);
+    case TcDownDgrad: return launch_kind<TcDownDgrad>(maps, prm, grid, mask, s, launches);
+    case TcDownWgrad: return launch_kind<TcDownWgrad>(maps, prm, grid, mask, s, launches);
+    case TcUpGateDgrad: return launch_kind<TcUpGateDgrad>(maps, prm, grid, mask, s, launches);
+    case TcUpGateWgrad: return launch_kind<TcUpGateWgrad>(maps, prm, grid, mask, s, launches);
     }
     return cudaErrorInvalidValue;
 }

@@ -10,6 +10,7 @@ namespace modse {
 // Host-side state owned by a layer object.
 struct TcPlan {
     int sm_count = 0;   // number of SMs of the device the layer last ran on
+    int tile_mask = -1; // which kernel variant runs each product (layout of tc_pair_mask()); -1: the process-wide default
 };
 
 // Process-wide debugging switch: run bf16 layers through the fp32-FMA grouped

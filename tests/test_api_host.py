@@ -102,3 +102,17 @@ def test_noise_gate_argument_errors_need_no_gpu():
     assert lib.modse_set_noise_grads(None, 0x1000, 0x1000) == B.MODSE_ERR_INVALID_ARG
     assert lib.modse_set_noise_grads(layer._h, 0x1000, 0x1000) == B.MODSE_OK
     layer.destroy()
+
+
+def test_tile_plan_validation_needs_no_gpu():
+    layer = B.ModseLayer(2048, [2816, 8448], 2)
+    assert layer.tile_plan() == -1                      # library default until tuned or set
+    layer.set_tile_plan(0x3A00)
+    assert layer.tile_plan() == 0x3A00
+    layer.set_tile_plan(-1)
+    assert layer.tile_plan() == -1
+    for bad in (-2, 0x4000, 0x40):
+        with pytest.raises(B.ModseError) as ei:
+            layer.set_tile_plan(bad)
+        assert ei.value.status == B.MODSE_ERR_INVALID_ARG
+    layer.destroy()

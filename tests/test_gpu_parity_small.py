@@ -191,3 +191,35 @@ def test_bf16_results_are_bitwise_reproducible_and_independent_of_tile_shape():
         assert np.array_equal(a[k], b[k]), k
         assert np.array_equal(a[k], c[k]), k
         assert np.array_equal(a[k], e[k]), k
+
+
+def test_tuned_plan_gives_identical_results():
+    """modse_tune_forward may pick another tile shape for the forward products; y must not change by a bit,
+    and the workspace it leaves must serve a backward pass."""
+    import torch
+    from paper_2409_12210_b200 import binding as B
+    cfg = dataclasses.replace(I.CONFIGS["train_16k"], name="tune_small", n_tokens=2048, d_model=512,
+                              ffn_sizes=(256, 768, 384, 640, 512, 512, 320, 704), seed=5)
+    inp, _ = H.screened(cfg)
+    dev, dt = "cuda", torch.bfloat16
+    layer = B.ModseLayer(cfg.d_model, cfg.ffn_sizes, cfg.top_k)
+    wr, wg, wu, wd = B.pack_weights(inp, dev)
+    x = torch.from_numpy(inp.x).to(dev, dt); dy = torch.from_numpy(inp.dy).to(dev, dt)
+    y0, y1 = torch.empty_like(x), torch.empty_like(x)
+    ws = layer.alloc_workspace(dt, x.shape[0], True)
+    layer.forward(wr, wg, wu, wd, x, y0, ws, True)
+    assert layer.tile_plan() == -1
+    plan = layer.tune_forward(wr, wg, wu, wd, x, y1, ws, True)
+    assert plan >= 0 and (plan & ~0x3F3F) == 0 and layer.tile_plan() == plan
+    assert torch.equal(y0, y1)
+    dx = torch.empty_like(x); dwr = torch.empty(wr.shape, dtype=torch.float32, device=dev)
+    dwg, dwu, dwd = (torch.empty_like(w) for w in (wg, wu, wd))
+    layer.backward(wr, wg, wu, wd, x, dy, dx, dwr, dwg, dwu, dwd, ws)      # the tuned forward was a saved one
+    dx_tuned = dx.clone()
+    layer.set_tile_plan(-1)
+    layer.forward(wr, wg, wu, wd, x, y1, ws, True)
+    layer.backward(wr, wg, wu, wd, x, dy, dx, dwr, dwg, dwu, dwd, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(y0, y1) and torch.equal(dx, dx_tuned)
+    assert layer.check_device_status(ws) == 0
+    layer.destroy()
