@@ -158,6 +158,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// `nboxes` 64-row boxes stacked from row y on (K-major operand): pairs of them go as one 128-row copy.
+__device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap *m64, const CUtensorMap *m128, uint32_t bar,
+                                              int x, int y, int nboxes)
+{
+    int i = 0;
+    for (; i + 2 <= nboxes; i += 2) tma_load_2d(dst + i * kBoxBytes, m128, bar, x, y + 64 * i);
+    if (i < nboxes) tma_load_2d(dst + i * kBoxBytes, m64, bar, x, y + 64 * i);
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -284,18 +293,15 @@ __device__ __forceinline__ void issue_loads(const TcMaps &maps, const Tile &t, i
                                             uint32_t bar)
 {
     if constexpr (KIND == TcUpGate) {
-        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, &maps.xp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        tma_load_rows(a_dst, &maps.xp, &maps.xp128, bar, kb * 64, t.prow0 + t.m0, 2);
         const int nb = t.ncols / 64;
-        for (int i = 0; i < nb; ++i) tma_load_2d(b_dst + i * kBoxBytes, &maps.wgate, bar, kb * 64, t.ho + t.n0 + 64 * i);
-        for (int i = 0; i < nb; ++i)
-            tma_load_2d(b_dst + (nb + i) * kBoxBytes, &maps.wup, bar, kb * 64, t.ho + t.n0 + 64 * i);
+        tma_load_rows(b_dst, &maps.wgate, &maps.wgate128, bar, kb * 64, t.ho + t.n0, nb);
+        tma_load_rows(b_dst + nb * kBoxBytes, &maps.wup, &maps.wup128, bar, kb * 64, t.ho + t.n0, nb);
     } else if constexpr (KIND == TcDown) {
-        for (int i = 0; i < 2; ++i)
-            tma_load_2d(a_dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + kb * t.cp + t.m0 + 64 * i);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + kb * 64, t.n0 + 64 * i);
+        tma_load_rows(a_dst, &maps.hm, &maps.hm128, bar, 0, t.pbase + kb * t.cp + t.m0, 2);
+        tma_load_rows(b_dst, &maps.wdown, &maps.wdown128, bar, t.ho + kb * 64, t.n0, t.b_boxes);
     } else if constexpr (KIND == TcDownDgrad) {
-        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, &maps.dyp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        tma_load_rows(a_dst, &maps.dyp, &maps.dyp128, bar, kb * 64, t.prow0 + t.m0, 2);
         for (int i = 0; i < t.b_boxes; ++i)
             tma_load_2d(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + 64 * i, kb * 64);
     } else if constexpr (KIND == TcDownWgrad) {
@@ -306,9 +312,9 @@ __device__ __forceinline__ void issue_loads(const TcMaps &maps, const Tile &t, i
         const int half = t.h / 64;
         const bool second = kb >= half;
         const int kk = second ? kb - half : kb;
-        const CUtensorMap *am = second ? &maps.db : &maps.da;
         const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
-        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + kk * t.cp + t.m0 + 64 * i);
+        tma_load_rows(a_dst, second ? &maps.db : &maps.da, second ? &maps.db128 : &maps.da128, bar, 0,
+                      t.pbase + kk * t.cp + t.m0, 2);
         for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(b_dst + i * kBoxBytes, bm, bar, t.n0 + 64 * i, t.ho + kk * 64);
     } else {
         const CUtensorMap *am = t.which ? &maps.db : &maps.da;
@@ -1169,20 +1175,19 @@ template <int KIND>
 __device__ __forceinline__ void load_rows(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
 {
     if constexpr (KIND == TcUpGate) {
-        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.xp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        tma_load_rows(dst, &maps.xp, &maps.xp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
     } else if constexpr (KIND == TcDown) {
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d(dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + kb * t.cp + t.m0 + 64 * i);
+        tma_load_rows(dst, &maps.hm, &maps.hm128, bar, 0, t.pbase + kb * t.cp + t.m0, t.a_boxes);
     } else if constexpr (KIND == TcDownDgrad) {
-        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.dyp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
+        tma_load_rows(dst, &maps.dyp, &maps.dyp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
     } else if constexpr (KIND == TcDownWgrad) {
         for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
     } else if constexpr (KIND == TcUpGateDgrad) {
         const int half = t.h / 64;
         const bool second = kb >= half;
         const int kk = second ? kb - half : kb;
-        const CUtensorMap *am = second ? &maps.db : &maps.da;
-        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, am, bar, 0, t.pbase + kk * t.cp + t.m0 + 64 * i);
+        tma_load_rows(dst, second ? &maps.db : &maps.da, second ? &maps.db128 : &maps.da128, bar, 0,
+                      t.pbase + kk * t.cp + t.m0, t.a_boxes);
     } else {
         const CUtensorMap *am = t.which ? &maps.db : &maps.da;
         for (int i = 0; i < t.a_boxes; ++i)
@@ -1196,10 +1201,10 @@ __device__ __forceinline__ void load_cols(const TcMaps &maps, const Tile &t, int
 {
     if constexpr (KIND == TcUpGate) {
         const int nb = t.ncols / 64;
-        for (int i = 0; i < nb; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wgate, bar, kb * 64, t.ho + t.n0 + 64 * i);
-        for (int i = 0; i < nb; ++i) tma_load_2d(dst + (nb + i) * kBoxBytes, &maps.wup, bar, kb * 64, t.ho + t.n0 + 64 * i);
+        tma_load_rows(dst, &maps.wgate, &maps.wgate128, bar, kb * 64, t.ho + t.n0, nb);
+        tma_load_rows(dst + nb * kBoxBytes, &maps.wup, &maps.wup128, bar, kb * 64, t.ho + t.n0, nb);
     } else if constexpr (KIND == TcDown) {
-        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wdown, bar, t.ho + kb * 64, t.n0 + 64 * i);
+        tma_load_rows(dst, &maps.wdown, &maps.wdown128, bar, t.ho + kb * 64, t.n0, t.b_boxes);
     } else if constexpr (KIND == TcDownDgrad) {
         for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + 64 * i, kb * 64);
     } else if constexpr (KIND == TcDownWgrad) {
@@ -1415,14 +1420,14 @@ EncodeTiledFn get_encode()
     return fn;
 }
 
-// bf16 row-major matrix [rows, cols] seen as a 2-D tensor, 64 x 64 boxes, 128-byte swizzle.
-bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols)
+// bf16 row-major matrix [rows, cols] seen as a 2-D tensor, boxes of 64 columns x box_rows rows, 128-byte swizzle.
+bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows = 64)
 {
     EncodeTiledFn fn = get_encode();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {64, 64};
+    const cuuint32_t box[2] = {64, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1436,19 +1441,22 @@ bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsP
 {
     const uint64_t panel_rows = L.hb / 64;
     bool ok = true;
-    ok = ok && encode_2d(&maps.xp, p.xp, L.Pmax, m.d);
-    ok = ok && encode_2d(&maps.wgate, w->w_gate, m.S, m.d);
-    ok = ok && encode_2d(&maps.wup, w->w_up, m.S, m.d);
-    ok = ok && encode_2d(&maps.wdown, w->w_down, m.d, m.S);
-    ok = ok && encode_2d(&maps.hm, p.hm, panel_rows, 64);
+    auto both = [&](CUtensorMap *m64, CUtensorMap *m128, const void *base, uint64_t rows, uint64_t cols) {
+        ok = ok && encode_2d(m64, base, rows, cols, 64) && encode_2d(m128, base, rows, cols, 128);
+    };
+    both(&maps.xp, &maps.xp128, p.xp, L.Pmax, m.d);
+    both(&maps.wgate, &maps.wgate128, w->w_gate, m.S, m.d);
+    both(&maps.wup, &maps.wup128, w->w_up, m.S, m.d);
+    both(&maps.wdown, &maps.wdown128, w->w_down, m.d, m.S);
+    both(&maps.hm, &maps.hm128, p.hm, panel_rows, 64);
     if (backward) {
-        ok = ok && encode_2d(&maps.dyp, p.dyp, L.Pmax, m.d);
-        ok = ok && encode_2d(&maps.da, p.da, panel_rows, 64);
-        ok = ok && encode_2d(&maps.db, p.db, panel_rows, 64);
+        both(&maps.dyp, &maps.dyp128, p.dyp, L.Pmax, m.d);
+        both(&maps.da, &maps.da128, p.da, panel_rows, 64);
+        both(&maps.db, &maps.db128, p.db, panel_rows, 64);
     } else {
-        maps.dyp = maps.xp;
-        maps.da = maps.hm;
-        maps.db = maps.hm;
+        maps.dyp = maps.xp;   maps.dyp128 = maps.xp128;
+        maps.da = maps.hm;    maps.da128 = maps.hm128;
+        maps.db = maps.hm;    maps.db128 = maps.hm128;
     }
     return ok;
 }

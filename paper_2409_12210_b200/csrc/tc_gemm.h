@@ -32,9 +32,12 @@ enum TcKind : int {
     TcUpGateWgrad = 5   // dWg = dA^T xp, dWu = dB^T xp
 };
 
-// Tensor maps of every TMA-loaded buffer (bf16, 64 x 64 boxes, 128-byte swizzle).
+// Tensor maps of every TMA-loaded buffer (bf16, 64 x 64 boxes, 128-byte swizzle), and the same tensors
+// with boxes of 128 rows: where an operand's rows are contiguous (K-major operands), one 16 KB copy fills
+// what two 8 KB copies would, in the same shared-memory layout, and the larger copies measured faster.
 struct TcMaps {
     CUtensorMap xp, dyp, wgate, wup, wdown, hm, da, db;
+    CUtensorMap xp128, dyp128, wgate128, wup128, wdown128, hm128, da128, db128;
 };
 
 bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
