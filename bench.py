@@ -45,6 +45,8 @@ NCU_TRAFFIC = {
 
 
 def ncu_traffic(stage: str, workload: str):
+    """DRAM bytes per launch from the committed ncu capture; None once the kernel source has changed since
+    (the caller also drops it when a tile plan other than the captured default is in use)."""
     import hashlib
     try:
         src = os.path.join(ROOT, "paper_2409_12210_b200", "csrc", "tc_gemm.cu")
@@ -417,7 +419,7 @@ def main():
     dom = max(stages, key=lambda s: s["ms"])
     roofline = {"kernel": dom["stage"], "bound": dom["bound"], "achieved": dom["achieved"],
                 "peak": pk["bf16_tflops_sustained"] if dom["bound"] == "tensor" else pk["hbm_gbs"],
-                "unit": dom["unit"], "frac": dom["frac"], "traffic": ncu_traffic(dom["stage"], cfg.name),
+                "unit": dom["unit"], "frac": dom["frac"], "traffic": ncu_traffic(dom["stage"], cfg.name) if tile_plan in (-1, 0x3A00) else None,
                 "traffic_unit": "bytes per launch (ncu dram read + write)", "peak_source": f"of {pk_src}",
                 "ms_per_launch": dom["ms"]}
 
