@@ -58,6 +58,16 @@ def ncu_traffic(stage: str, workload: str):
     return NCU_TRAFFIC["bytes_per_launch"].get(stage)
 
 
+def same_kernel_as_captured(stage: str, tile_plan: int) -> bool:
+    """True if `tile_plan` runs `stage` on the kernel variant of the ncu capture (the library's default plan)."""
+    kinds = {"upgate_gemm_swiglu": 0, "down_gemm": 1, "down_dgrad_swiglu_bwd": 2, "down_wgrad": 3,
+             "upgate_dgrad": 4, "upgate_wgrad": 5}
+    if tile_plan < 0 or stage not in kinds:
+        return True
+    k, default = kinds[stage], 0x3A00
+    return ((tile_plan >> k) & 1) == ((default >> k) & 1) and ((tile_plan >> (8 + k)) & 1) == ((default >> (8 + k)) & 1)
+
+
 STAGE_BOUND = ["hbm", "hbm", "hbm", "tensor", "tensor", "hbm", "hbm", "tensor", "tensor", "tensor", "tensor", "hbm"]
 
 
@@ -419,7 +429,7 @@ def main():
     dom = max(stages, key=lambda s: s["ms"])
     roofline = {"kernel": dom["stage"], "bound": dom["bound"], "achieved": dom["achieved"],
                 "peak": pk["bf16_tflops_sustained"] if dom["bound"] == "tensor" else pk["hbm_gbs"],
-                "unit": dom["unit"], "frac": dom["frac"], "traffic": ncu_traffic(dom["stage"], cfg.name) if tile_plan in (-1, 0x3A00) else None,
+                "unit": dom["unit"], "frac": dom["frac"], "traffic": ncu_traffic(dom["stage"], cfg.name) if same_kernel_as_captured(dom["stage"], tile_plan) else None,
                 "traffic_unit": "bytes per launch (ncu dram read + write)", "peak_source": f"of {pk_src}",
                 "ms_per_launch": dom["ms"]}
 
