@@ -198,7 +198,7 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     inp = I.generate(cfg)
-    n_tok = args.cpu_tokens
+    n_tok = args.ref_tokens
     for _ in range(args.warmup if args.warmup < 2 else 1):
         cpu_oracle_sample(inp, n_tok)
     times, cores = [], 1
@@ -226,7 +226,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="train_16k", choices=sorted(I.CONFIGS))
-    ap.add_argument("--cpu-tokens", type=int, default=64, help="tokens of the CPU baseline sample")
+    ap.add_argument("--cpu-tokens", type=int, default=256, help="tokens of the CPU baseline sample (about 15 s on 16 cores)")
+    ap.add_argument("--ref-tokens", type=int, default=64,
+                    help="--impl reference: tokens of the sample each step times (about 4 s on 16 cores)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tokens", type=int, default=None, help="override the workload's token count")
     ap.add_argument("--layers", type=int, default=1,
