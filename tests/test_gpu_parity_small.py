@@ -162,9 +162,10 @@ def test_bf16_empty_expert_gets_zero_weight_gradients():
     assert np.all(gpu["dw_down"][:, h0:h1] == 0)
 
 
-@pytest.mark.parametrize("n_experts", [16, 40])
+@pytest.mark.parametrize("n_experts", [16, 40, 256])
 def test_bf16_many_experts(n_experts):
-    # 16 experts: two 8-expert tiles in the tensor-core router; 40: the general fp32-FMA router
+    # 16 experts: two 8-expert tiles in the tensor-core router; 40: the general fp32-FMA router;
+    # 256: the largest number of experts the library accepts (about 23 assignments per expert)
     rng = np.random.default_rng(n_experts)
     widths = tuple(int(w) for w in rng.choice([64, 128, 192, 256], n_experts))
     cfg = I.LayerConfig(f"bf16_N{n_experts}", "bf16", 256, widths, 2, 3000, seed=n_experts, weight_std=0.05)
@@ -223,3 +224,16 @@ def test_tuned_plan_gives_identical_results():
     assert torch.equal(y0, y1) and torch.equal(dx, dx_tuned)
     assert layer.check_device_status(ws) == 0
     layer.destroy()
+
+
+def test_f32_maximum_number_of_experts():
+    """256 experts (the library's limit), fp32 path: every table and every gradient against the oracle."""
+    rng = np.random.default_rng(256)
+    widths = tuple(int(w) for w in rng.choice([16, 32, 48], 256))
+    cfg = I.LayerConfig("f32_N256", "f32", 64, widths, 2, 1500, seed=256)
+    inp, _ = H.screened(cfg)
+    gpu = H.run_gpu(inp, True)
+    H.check_all(inp, gpu, H.run_oracle(inp, True), 1e-4)
+    with pytest.raises(Exception):
+        from paper_2409_12210_b200 import binding as B
+        B.ModseLayer(64, (16,) * 257, 2)
