@@ -122,7 +122,8 @@ def test_small_bf16_forward_only_without_saving():
 
 
 @pytest.mark.parametrize("T,k,widths,d", [(1, 2, (64, 128), 128), (129, 1, (64, 192, 128), 128),
-                                          (700, 2, (448, 64, 320, 192), 384)])
+                                          (700, 2, (448, 64, 320, 192), 384),
+                                          (600, 2, (128, 320, 64, 192, 256, 64, 128, 192), 4096)])   # wide model: 64 k-blocks
 def test_bf16_degenerate_and_ragged_shapes(T, k, widths, d):
     # With a handful of tokens per expert the weight gradients are sums of a few outer products:
     # so heavy-tailed that max|err|/RMS says nothing (one bf16 operand rounding of the largest
