@@ -70,7 +70,7 @@ constexpr int kThreads = 320;                   // TMA warp, MMA warp, eight epi
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
-constexpr int kEpiRowBytes = 64 + 16;            // a 32-element bf16 chunk of one row, skewed by 16 bytes
+constexpr int kEpiRowBytes = 64;                 // a 32-element bf16 chunk of one row; 16-byte pieces XOR-swizzled
 constexpr int kEpiWarpBytes = 32 * kEpiRowBytes;
 
 struct TcParams {
@@ -344,18 +344,22 @@ __device__ __forceinline__ void issue_loads(const TcMaps &maps, const Tile &t, i
 // afterwards four neighbouring lanes cover the 64 bytes of one row and an instruction moves eight
 // whole 64-byte row segments.  `own` points at this thread's own row chunk.
 // rows_valid: rows of this warp (0..32, counted from the warp's first row) that may be written.
+// Byte offset of 16-byte piece q of row r in a warp's staging buffer.  Rows are 64 bytes; the piece index is
+// XORed with (r / 2) % 4, so that both access patterns are free of bank conflicts: eight lanes writing the
+// same piece of eight consecutive rows, and eight lanes reading all pieces of two consecutive rows.
+__device__ __forceinline__ int epi_piece(int r, int q) { return r * kEpiRowBytes + ((q ^ ((r >> 1) & 3)) << 4); }
+
 __device__ __forceinline__ void store_u4x4_staged(unsigned char *stg, int lane, unsigned char *own, long long row_stride_bytes,
                                                   const uint4 (&w)[4], int rows_valid)
 {
-    uint4 *mine = reinterpret_cast<uint4 *>(stg + lane * kEpiRowBytes);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) mine[q] = w[q];
+    for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4 *>(stg + epi_piece(lane, q)) = w[q];
     __syncwarp();
     const int q = lane & 3;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int rr = 8 * j + (lane >> 2);
-        const uint4 val = *reinterpret_cast<const uint4 *>(stg + rr * kEpiRowBytes + q * 16);
+        const uint4 val = *reinterpret_cast<const uint4 *>(stg + epi_piece(rr, q));
         if (rr < rows_valid) *reinterpret_cast<uint4 *>(own + (long long)(rr - lane) * row_stride_bytes + q * 16) = val;
     }
     __syncwarp();
@@ -412,12 +416,11 @@ __device__ __forceinline__ void untranspose_rows(unsigned char *stg, int lane, c
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const int rr = 8 * j + (lane >> 2);
-        *reinterpret_cast<uint4 *>(stg + rr * kEpiRowBytes + q * 16) = raw[j];
+        *reinterpret_cast<uint4 *>(stg + epi_piece(rr, q)) = raw[j];
     }
     __syncwarp();
-    const uint4 *mine = reinterpret_cast<const uint4 *>(stg + lane * kEpiRowBytes);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) own[i] = mine[i];
+    for (int i = 0; i < 4; ++i) own[i] = *reinterpret_cast<const uint4 *>(stg + epi_piece(lane, i));
     __syncwarp();
 }
 
