@@ -38,9 +38,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # profiles/tc_grouped_gemm_train_16k_ncu_full.md; valid only for that workload and for the kernel source it was
 # taken from (first 16 hex digits of the SHA-256 of csrc/tc_gemm.cu), otherwise "traffic" is reported as null.
 NCU_TRAFFIC = {
-    "workload": "train_16k", "tc_gemm_sha256_16": "c6bd8a29bb70cd7a",
-    "bytes_per_launch": {"upgate_gemm_swiglu": 1.589e9, "down_gemm": 0.922e9, "down_dgrad_swiglu_bwd": 1.945e9,
-                         "down_wgrad": 0.741e9, "upgate_dgrad": 1.909e9, "upgate_wgrad": 1.329e9},
+    "workload": "train_16k", "tc_gemm_sha256_16": "c818e5c311c654cd",
+    "bytes_per_launch": {"upgate_gemm_swiglu": 1.591e9, "down_gemm": 0.932e9, "down_dgrad_swiglu_bwd": 1.953e9,
+                         "down_wgrad": 0.753e9, "upgate_dgrad": 1.910e9, "upgate_wgrad": 1.310e9},
 }
 
 

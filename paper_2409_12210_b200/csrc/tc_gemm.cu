@@ -238,6 +238,45 @@ template <> struct KindTraits<TcDownWgrad>   { static constexpr bool a_mn = true
 template <> struct KindTraits<TcUpGateDgrad> { static constexpr bool a_mn = false, b_mn = true; };
 template <> struct KindTraits<TcUpGateWgrad> { static constexpr bool a_mn = true,  b_mn = true; };
 
+// Row block and column block of tile `local` of an expert with mt x nt tiles.
+//   N_FASTEST: the column blocks of one row block are consecutive.
+//   otherwise: the row blocks of one column block are consecutive, within groups of row blocks that hold at
+//   most `rows_per_group` row tiles.  Without the groups an expert with many tokens streams all of its rows
+//   once per column block (67 MB of xp per column block at 16 K rows: L2 keeps neither the rows nor the
+//   column operand); with them a group's rows stay in L2 while its column blocks go by.  Groups are of
+//   equal size (+-1 row tile), so that no group is too small to share the column operand.
+template <bool N_FASTEST>
+__device__ __forceinline__ void tile_coords(int local, int mt, int nt, int rows_per_group, int &mb, int &nb)
+{
+    if constexpr (N_FASTEST) {
+        mb = local / nt;
+        nb = local % nt;
+    } else {
+        const int n_g = (mt + rows_per_group - 1) / rows_per_group;
+        if (n_g <= 1) {
+            mb = local % mt;
+            nb = local / mt;
+            return;
+        }
+        const int base = mt / n_g, extra = mt % n_g;
+        const int big = (base + 1) * nt;              // tiles of each of the first `extra` groups
+        int rem, rows, row0;
+        if (local < extra * big) {
+            const int g = local / big;
+            rem = local - g * big; rows = base + 1; row0 = g * (base + 1);
+        } else {
+            const int l2 = local - extra * big;
+            const int g = l2 / (base * nt);
+            rem = l2 - g * base * nt; rows = base; row0 = extra * (base + 1) + g * base;
+        }
+        mb = row0 + rem % rows;
+        nb = rem / rows;
+    }
+}
+
+// Rows of the row operand that one group may hold: 16 M elements (32 MB of bf16) across the model width.
+__device__ __forceinline__ int group_row_tiles(int d, int tile_rows) { return max(1, ((16 << 20) / d) / tile_rows); }
+
 struct Tile {
     int e, cp, h, ho, prow0, pbase;   // expert, padded rows, width, width offset, first padded row, first panel row
     int m0, n0, mrows, ncols, nk, which;
@@ -277,8 +316,8 @@ __device__ __forceinline__ Tile decode_tile(const TcParams &prm, const SmemTail 
     // panels of the down wgrad), column-block fastest where all column blocks of one row block
     // fit in flight at once (d / 256 = 8 column blocks), so the row operand is read once.
     constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
-    const int mb = n_fastest ? local / nt : local % mt;
-    const int nb = n_fastest ? local % nt : local / mt;
+    int mb, nb;
+    tile_coords<n_fastest>(local, mt, nt, group_row_tiles(d, 128), mb, nb);
     t.nk = nk;
     t.which = 0;
     t.mrows = 128;
@@ -851,8 +890,8 @@ __device__ __forceinline__ Tile decode_tile2(const TcParams &prm, const SmemTail
     expert_shape2<KIND>(t.cp, t.h, d, mt, nt, nk);
     const int local = tile - st->tstart[cursor];
     constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
-    int mb = n_fastest ? local / nt : local % mt;
-    const int nb = n_fastest ? local % nt : local / mt;
+    int mb, nb;
+    tile_coords<n_fastest>(local, mt, nt, group_row_tiles(d, 256), mb, nb);
     t.nk = nk;
     t.which = 0;
     int row_extent;                       // extent of the tile's row dimension for this expert
@@ -1157,8 +1196,8 @@ __device__ __forceinline__ Tile decode_tile_wide(const TcParams &prm, const Smem
     expert_shape_wide<KIND>(t.cp, t.h, d, mt, nt, nk);
     const int local = tile - st->tstart[cursor];
     constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
-    int mb = n_fastest ? local / nt : local % mt;
-    const int nb = n_fastest ? local % nt : local / mt;
+    int mb, nb;
+    tile_coords<n_fastest>(local, mt, nt, group_row_tiles(d, 256), mb, nb);
     t.nk = nk;
     t.which = 0;
     int row_extent;
