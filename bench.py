@@ -153,12 +153,17 @@ class ClockSampler:
             self.thread.join(timeout=1.0)
         if not self.rows:
             return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": [self.err or "no samples"]}
-        bits = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
+        bits = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+                0x2: "applications_clocks_setting", 0x10: "sync_boost", 0x80: "hw_power_brake_slowdown",
+                0x100: "display_clock_setting"}                # 0x1 (gpu_idle) is not a limit and is left out
         seen = set()
         for _, r, _ in self.rows:
             for b, name in bits.items():
                 if r & b:
                     seen.add(name)
+            other = r & ~(sum(bits) | 0x1)
+            if other:
+                seen.add(f"other:0x{other:x}")
         return {"sm_mhz": float(np.median([r[0] for r in self.rows])), "sm_max_mhz": self.max_sm,
                 "power_w_max": max(r[2] for r in self.rows), "samples": len(self.rows), "reasons": sorted(seen)}
 
