@@ -165,6 +165,7 @@ class ClockSampler:
             if other:
                 seen.add(f"other:0x{other:x}")
         return {"sm_mhz": float(np.median([r[0] for r in self.rows])), "sm_max_mhz": self.max_sm,
+                "sm_mhz_range": [min(r[0] for r in self.rows), max(r[0] for r in self.rows)],
                 "power_w_max": max(r[2] for r in self.rows), "samples": len(self.rows), "reasons": sorted(seen)}
 
 
