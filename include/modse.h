@@ -144,8 +144,20 @@ modse_status_t modse_get_gate_grads(const modse_layer_t *layer, const void *work
                                     const float **dg, const float **dz);
 
 /* Synchronises the stream and reads the status word kernels write when a
- * bounded wait expires or an index check fails; MODSE_OK if none did.        */
+ * bounded wait expires (MODSE_ERR_DEVICE_TIMEOUT) or an index check fails
+ * (MODSE_ERR_DEVICE_BOUNDS); MODSE_OK if none did.  The word is cleared by the
+ * next modse_forward.  Index checks are always on: every kernel that follows a
+ * row or token index read from the routing tables compares it with the table's
+ * extent first and skips the access if it lies outside.
+ *
+ * modse_set_debug_checks(layer, 1) (or the environment variable MODSE_DEBUG=1
+ * at modse_create) adds guard blocks: every region of the workspace is followed
+ * by 256 spare bytes whose head modse_forward fills with a pattern and this
+ * call compares; a kernel that wrote past its region turns up as
+ * MODSE_ERR_DEVICE_BOUNDS.  (The blocks are part of modse_workspace_bytes in
+ * either mode.)  No counterpart in the paper.                                */
 modse_status_t modse_check_device_status(modse_layer_t *layer, const void *workspace, void *cuda_stream);
+modse_status_t modse_set_debug_checks(modse_layer_t *layer, int on);
 
 /* Number of kernel launches the last forward/backward call on this layer
  * enqueued (for launch accounting in benchmarks).                            */
@@ -185,14 +197,35 @@ modse_status_t modse_set_output_f32(modse_layer_t *layer, int on);
  * the layer object for all later calls.  It allocates no device memory, SYNCHRONISES the stream, and leaves y
  * and the workspace as one modse_forward would.  Results do not depend on the plan (the K order of every sum
  * is the same).  fp32 layers have one kernel shape: the call returns MODSE_OK at once.
- * modse_get_tile_plan returns the plan (-1: library default; else bit k: product k on the two-SM kernel,
- * bit 8+k: product k on the 256-row kernel, k = 0 up/gate, 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate
- * dgrad, 5 up/gate wgrad); modse_set_tile_plan installs one (e.g. a plan found earlier on the same device). */
+ * modse_get_tile_plan returns the plan (-1: library default; else bit k set: product k on 256-row tiles,
+ * clear: on 128-row tiles; k = 0 up/gate, 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate dgrad, 5 up/gate
+ * wgrad); modse_set_tile_plan installs one (e.g. a plan found earlier on the same device). */
 modse_status_t modse_tune_forward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
                                   const void *x, int n_tokens, void *y, void *workspace, size_t workspace_bytes,
                                   int save_for_backward, void *cuda_stream);
 int modse_get_tile_plan(const modse_layer_t *layer);
 modse_status_t modse_set_tile_plan(modse_layer_t *layer, int plan);
+
+/* Fusions across the permutation (bf16 layers; Sec. 2 Eq. 1 and Sec. 3.1 Eq. 4 say "select the top-k experts
+ * and combine their outputs" and fix no intermediate buffers).  `flags` is a sum of
+ *   MODSE_FUSE_GATHER   the up/gate product gathers its rows from x through the permutation (TMA row gather)
+ *                       instead of reading the grouped copy of x; a forward that saves nothing for backward
+ *                       then skips the permute kernel altogether;
+ *   MODSE_FUSE_DG_ROWDOT  the gate gradient dg[t,j] = <dY_t W_down_e, Hm_row> / g is accumulated inside the
+ *                       down-dgrad epilogue (one partial per 128 columns, summed in column order), so
+ *                       backward no longer reads the fp32 expert outputs o;
+ *   MODSE_FUSE_SCATTER  with fp32 outputs (modse_set_output_f32) and top_k <= 2: the down product adds its
+ *                       rows straight into y and the up/gate dgrad into dx (both zeroed first; two addends
+ *                       into a zeroed element commute, so the result is the same bits in any order), the
+ *                       buffers o and dxp and the combine pass disappear; implies MODSE_FUSE_DG_ROWDOT.
+ * A flag that does not apply to a call (fp32 layer, bf16 outputs, top_k > 2) is ignored by that call.
+ * A backward call follows the forward call it belongs to.  Results: GATHER and SCATTER give the same bits as
+ * the unfused path; DG_ROWDOT sums dg in another order (same tolerance).  Default: none.              */
+#define MODSE_FUSE_GATHER 1
+#define MODSE_FUSE_DG_ROWDOT 2
+#define MODSE_FUSE_SCATTER 4
+modse_status_t modse_set_fusion(modse_layer_t *layer, int flags);
+int modse_get_fusion(const modse_layer_t *layer);
 
 /* Second term of the router logits (Sec. 2, Eq. 2 with the RMSNorm and Softplus
  * definitions that follow it):
@@ -240,12 +273,20 @@ modse_status_t modse_set_noise_grads(modse_layer_t *layer, float *dw_noise, floa
  * All calls share the one array and it keeps the last call's contents (the
  * call clears what must start at zero): two calls that overlap on the GPU -
  * different streams, or different host threads - race on it; serialise them.
- * Calls no cudaMalloc/cudaFree and no allocating library routine.            */
+ * Calls no cudaMalloc/cudaFree and no allocating library routine.
+ * The array's device address is cached per process and per device context:
+ * serialise the first calls of several host threads, and do not use the
+ * library across a cudaDeviceReset.
+ * modse_route_static_scratch_status synchronises `cuda_stream` and returns what
+ * the kernels of the last call on the current device recorded in the array's
+ * status word (MODSE_OK, MODSE_ERR_DEVICE_BOUNDS, MODSE_ERR_DEVICE_TIMEOUT);
+ * it plays the part of modse_check_device_status, which needs a workspace.   */
 modse_status_t modse_route_static_scratch(modse_dtype_t dtype, int d_model, int n_experts, int top_k,
                                           const void *x, const void *w_router, int n_tokens, int *topk_idx,
                                           float *topk_gate, int *counts, int *counts_slot, int *offsets,
                                           int *row_of, int *token_of, void *cuda_stream);
 size_t modse_route_static_scratch_capacity(void);
+modse_status_t modse_route_static_scratch_status(void *cuda_stream);
 
 /* Per-stage device timing (profiling aid).  After modse_stage_timing_begin the
  * next max_calls forward/backward calls on this layer bracket each of their
@@ -267,14 +308,29 @@ const char *modse_stage_name(int stage);
  * be called with save_for_backward = 1.  Off by default.                    */
 void modse_debug_use_fma_path(int on);
 
-/* Tuning aid, process-wide: which of three tile shapes each grouped product k
- * (0 up/gate, 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate dgrad, 5 up/gate
- * wgrad) runs on.  Bit k of `mask`: 256-row tiles on pairs of SMs
- * (cta_group::2); bit 8+k: 256-row tiles on one SM (two accumulators sharing
- * the column operand); neither: 128-row tiles on one SM.  The library's default
- * is bits 8+{1,3,4,5}.  Every choice gives bit-identical results (the order
- * in which each output element is summed does not depend on the tile shape). */
-void modse_debug_set_pair_kernels(int mask);
+/* Tuning aid, process-wide: the tile plan (see modse_get_tile_plan) of layers that have none of their own.
+ * The library's default puts products 1, 3, 4 and 5 on 256-row tiles.  Every choice gives bit-identical
+ * results (the order in which each output element is summed does not depend on the tile shape).        */
+void modse_debug_set_default_tile_plan(int plan);
+
+/* Tuning aid, process-wide: 1 (default) - the CTAs of a grouped product take tiles, longest K first, from a
+ * counter in the workspace; 0 - the tiles are dealt to the CTAs round-robin.  Same results either way.   */
+void modse_debug_set_dynamic_tiles(int on);
+
+/* Failure-path aids, process-wide.  Every wait inside a kernel gives up after a limit (default 2000 ms),
+ * records MODSE_ERR_DEVICE_TIMEOUT in the status word, lets its copies in flight land, frees its tensor
+ * memory and returns; modse_debug_set_wait_limit_ms changes the limit (1..60000).
+ * modse_debug_skip_tile_loads(product, tile) makes the CTA that is handed tile `tile` of grouped product
+ * `product` (0..5) issue no loads for it and stop producing, so that its consumers run into that limit with
+ * nothing in flight; (-1, -1) switches it off.  For tests of the time-out path on tiny inputs.          */
+void modse_debug_set_wait_limit_ms(int ms);
+void modse_debug_skip_tile_loads(int product, int tile);
+
+/* Test aid: byte offsets, inside a workspace of the given shape, of the padded row table prow_of [T,k] and of
+ * the guard block behind topk_idx, and the number of padded rows (the extent row indices are checked against). */
+modse_status_t modse_debug_workspace_offsets(const modse_layer_t *layer, modse_dtype_t dtype, int n_tokens,
+                                             int save_for_backward, size_t *prow_of_offset, size_t *first_guard_offset,
+                                             int *padded_rows);
 
 #ifdef __cplusplus
 }

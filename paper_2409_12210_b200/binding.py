@@ -24,6 +24,10 @@ MODSE_ERR_DEVICE_BOUNDS = 7
 MODSE_F32 = 0
 MODSE_BF16 = 1
 N_STAGES = 12
+MODSE_FUSE_GATHER = 1
+MODSE_FUSE_DG_ROWDOT = 2
+MODSE_FUSE_SCATTER = 4
+DEFAULT_TILE_PLAN = 0b111010       # products 1, 3, 4, 5 on 256-row tiles
 
 
 class ModseError(RuntimeError):
@@ -87,6 +91,8 @@ def load():
     lib.modse_route_static_scratch.restype = ci
     lib.modse_route_static_scratch.argtypes = [ci, ci, ci, ci, vp, vp, ci, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.modse_route_static_scratch_capacity.restype = sz
+    lib.modse_route_static_scratch_status.restype = ci
+    lib.modse_route_static_scratch_status.argtypes = [vp]
     lib.modse_aux_loss.restype = ci
     lib.modse_aux_loss.argtypes = [vp, vp, ci, ctypes.c_float, vp, vp, vp, vp]
     lib.modse_set_aux_loss.restype = ci
@@ -109,8 +115,22 @@ def load():
     lib.modse_stage_timing_end.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ip]
     lib.modse_stage_name.restype = ctypes.c_char_p
     lib.modse_stage_name.argtypes = [ci]
-    lib.modse_debug_set_pair_kernels.restype = None
-    lib.modse_debug_set_pair_kernels.argtypes = [ci]
+    lib.modse_debug_set_default_tile_plan.restype = None
+    lib.modse_debug_set_default_tile_plan.argtypes = [ci]
+    lib.modse_debug_set_dynamic_tiles.restype = None
+    lib.modse_debug_set_dynamic_tiles.argtypes = [ci]
+    lib.modse_debug_set_wait_limit_ms.restype = None
+    lib.modse_debug_set_wait_limit_ms.argtypes = [ci]
+    lib.modse_debug_skip_tile_loads.restype = None
+    lib.modse_debug_skip_tile_loads.argtypes = [ci, ci]
+    lib.modse_debug_workspace_offsets.restype = ci
+    lib.modse_debug_workspace_offsets.argtypes = [vp, ci, ci, ci, ctypes.POINTER(sz), ctypes.POINTER(sz), ip]
+    lib.modse_set_debug_checks.restype = ci
+    lib.modse_set_debug_checks.argtypes = [vp, ci]
+    lib.modse_set_fusion.restype = ci
+    lib.modse_set_fusion.argtypes = [vp, ci]
+    lib.modse_get_fusion.restype = ci
+    lib.modse_get_fusion.argtypes = [vp]
     lib.modse_debug_use_fma_path.restype = None
     lib.modse_debug_use_fma_path.argtypes = [ci]
     _lib = lib
@@ -148,12 +168,30 @@ def route_static_scratch(x, w_router, top_k: int):
     return out
 
 
+def route_static_scratch_status() -> int:
+    """Status word the last modse_route_static_scratch call on this device left (synchronises the stream)."""
+    import torch
+    return int(load().modse_route_static_scratch_status(ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)))
+
+
 def stage_name(i: int) -> str:
     return load().modse_stage_name(int(i)).decode()
 
 
-def debug_set_pair_kernels(mask: int) -> None:
-    load().modse_debug_set_pair_kernels(int(mask))
+def debug_set_default_tile_plan(plan: int) -> None:
+    load().modse_debug_set_default_tile_plan(int(plan))
+
+
+def debug_set_dynamic_tiles(on: bool) -> None:
+    load().modse_debug_set_dynamic_tiles(int(bool(on)))
+
+
+def debug_set_wait_limit_ms(ms: int) -> None:
+    load().modse_debug_set_wait_limit_ms(int(ms))
+
+
+def debug_skip_tile_loads(product: int, tile: int) -> None:
+    load().modse_debug_skip_tile_loads(int(product), int(tile))
 
 
 def debug_use_fma_path(on: bool) -> None:
@@ -288,6 +326,28 @@ class ModseLayer:
 
     def check_device_status(self, workspace) -> int:
         return int(load().modse_check_device_status(self._h, workspace.data_ptr(), self._stream()))
+
+    def set_debug_checks(self, on: bool) -> None:
+        st = load().modse_set_debug_checks(self._h, int(bool(on)))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_set_debug_checks")
+
+    def set_fusion(self, flags: int) -> None:
+        st = load().modse_set_fusion(self._h, int(flags))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_set_fusion")
+
+    def fusion(self) -> int:
+        return int(load().modse_get_fusion(self._h))
+
+    def debug_workspace_offsets(self, dtype_code: int, n_tokens: int, save_for_backward: bool):
+        """(byte offset of prow_of, byte offset of the guard block behind topk_idx, padded rows)."""
+        a, b, c = ctypes.c_size_t(0), ctypes.c_size_t(0), ctypes.c_int(0)
+        st = load().modse_debug_workspace_offsets(self._h, dtype_code, n_tokens, int(save_for_backward),
+                                                  ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+        if st != MODSE_OK:
+            raise ModseError(st, "modse_debug_workspace_offsets")
+        return int(a.value), int(b.value), int(c.value)
 
     def set_aux_loss(self, alpha: float) -> None:
         st = load().modse_set_aux_loss(self._h, float(alpha))

@@ -1,6 +1,7 @@
 // Host side of libmodse: argument checking, workspace carving and the order in
 // which the stages of the MoDSE layer are enqueued (see include/modse.h).
 #include <algorithm>
+#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -21,7 +22,10 @@ struct modse_layer {
     float aux_alpha = 0.f;        // coefficient of the auxiliary load-balance loss added to the objective in backward
     int out_f32 = 0;              // bf16 layers: write y, dx and expert weight gradients as fp32
     modse::NoiseGate noise;       // second term of the router logits (borrowed device pointers)
-    modse::TcPlan tc;             // device facts of the bf16 path
+    modse::TcPlan tc;             // device facts of the bf16 path, cached tensor maps
+    int fuse = 0;                 // kFuse* bits requested for this layer
+    int fwd_fuse = 0;             // bits the last forward ran with (backward follows them)
+    int debug_checks = 0;         // guard blocks between workspace regions are written and checked
     // optional per-stage device timing: events [call][stage][start/stop]
     std::vector<cudaEvent_t> ev;
     std::vector<unsigned char> ev_used;   // [call][stage]
@@ -45,7 +49,15 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
     for (int j = 0; j < m.k; ++j) topk_sum += (size_t)h_desc[j];
     L.hb = (size_t)T * topk_sum + (size_t)(kRowPad - 1) * m.S;
     size_t off = 0;
-    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.n_canary = 0;
+    // every region is followed by a 256-byte guard block (see kCanaryPattern)
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off = align_up(off + bytes, 256);
+        if (L.n_canary < kMaxCanaries) L.canary[L.n_canary++] = off;
+        off += 256;
+        return o;
+    };
     const size_t kT = (size_t)m.k * T, N = m.N;
     L.status = take(64);
     L.topk_idx = take(kT * 4);
@@ -79,6 +91,8 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
         L.da = take(L.hb * esz);
         L.db = take(L.hb * esz);
         L.dxp = take((size_t)L.Pmax * m.d * 4);   // fp32 for every layer type
+        L.dg_slots = 2 * ((h_desc[0] + 255) / 256);
+        L.dg_part = take((size_t)L.dg_slots * L.Pmax * 4);
     } else if (esz == 4) {
         // the fp32 path always materialises the two pre-activations
         L.a_pre = take(L.hb * esz);
@@ -114,6 +128,7 @@ WsPtrs carve(void *ws, const WsLayout &L)
     p.dg = (float *)(b + L.dg);
     p.dz = (float *)(b + L.dz);
     p.dwr_partial = (float *)(b + L.dwr_partial);
+    p.dg_part = (float *)(b + L.dg_part);
     p.xp = b + L.xp;
     p.a_pre = b + L.a_pre;
     p.b_pre = b + L.b_pre;
@@ -185,6 +200,8 @@ modse_layer_t *modse_create(int d_model, int n_experts, const int *ffn_sizes, in
     L->h.assign(ffn_sizes, ffn_sizes + n_experts);
     L->h_desc = L->h;
     std::sort(L->h_desc.begin(), L->h_desc.end(), [](int a, int b) { return a > b; });
+    const char *dbg = std::getenv("MODSE_DEBUG");
+    L->debug_checks = (dbg != nullptr && dbg[0] != '\0' && dbg[0] != '0') ? 1 : 0;
     return L;
 }
 
@@ -284,6 +301,34 @@ static modse_status_t check_common(const modse_layer_t *layer, modse_dtype_t dty
     return MODSE_OK;
 }
 
+// Tensor maps of a call: encoded once per (workspace, x, weights, token count, direction) and kept in the layer.
+static const TcMaps *cached_maps(modse_layer *layer, const LayerMeta &m, const WsLayout &L, const WsPtrs &p,
+                                 const modse_weights_t *w, const void *x, const void *ws, bool backward)
+{
+    TcMapKey key;
+    key.ws = ws; key.x = x; key.w_gate = w->w_gate; key.w_up = w->w_up; key.w_down = w->w_down;
+    key.T = L.T; key.backward = backward ? 1 : 0;
+    TcMaps &maps = backward ? layer->tc.maps_bwd : layer->tc.maps_fwd;
+    TcMapKey &have = backward ? layer->tc.key_bwd : layer->tc.key_fwd;
+    if (!(have == key)) {
+        have = TcMapKey{};
+        if (!tc_fill_maps(maps, m, L, p, w, x, backward)) return nullptr;
+        have = key;
+    }
+    return &maps;
+}
+
+// Fusions that apply to a call: scatter-adding epilogues need fp32 outputs of a bf16 layer on the tensor-core path
+// (two addends per element at most: top_k <= 2) and take dg from the row dot, since o is then never written.
+static int effective_fuse(const modse_layer *layer, modse_dtype_t dtype, bool of32)
+{
+    if (dtype != MODSE_BF16 || tc_force_simt()) return 0;
+    int f = layer->fuse & kFuseAll;
+    if (!of32 || layer->meta.k > 2) f &= ~kFuseScatter;
+    if (f & kFuseScatter) f |= kFuseDgRowdot;
+    return f;
+}
+
 modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
                              const void *x, int n_tokens, void *y, void *workspace, size_t workspace_bytes,
                              int save_for_backward, void *cuda_stream)
@@ -301,12 +346,16 @@ modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const mo
     layer->fwd_ws = nullptr;
     const bool of32 = dtype == MODSE_BF16 && layer->out_f32 != 0;
     if (of32 && tc_force_simt()) return MODSE_ERR_UNSUPPORTED;
+    const int fuse = effective_fuse(layer, dtype, of32);
 
     StageTimer tm(layer, s);
-    MODSE_CUDA(cudaMemsetAsync(p.status, 0, 64, s));
+    MODSE_CUDA(cudaMemsetAsync(p.status, 0, 64, s));           // status word and the tile counters
+    if (layer->debug_checks) MODSE_CUDA(launch_canaries(workspace, L, false, p.status, s));
     MODSE_STAGE(tm, 0, launch_router(dtype, m, x, weights->w_router, n_tokens, p, layer->noise, s, &launches));
     MODSE_STAGE(tm, 1, launch_rank(m, n_tokens, L.Pmax, p, s, &launches));
-    MODSE_STAGE(tm, 2, launch_permute(dtype, m, x, n_tokens, p, s, &launches));
+    // the grouped copy of x feeds the up/gate product (unless that gathers its rows itself) and its weight gradient
+    if (!(fuse & kFuseGather) || save)
+        MODSE_STAGE(tm, 2, launch_permute(dtype, m, x, n_tokens, L.Pmax, p, s, &launches));
     if (dtype == MODSE_F32 || tc_force_simt()) {
         // the bf16 cross-check path materialises both pre-activations, which only a saved forward has room for
         if (dtype == MODSE_BF16 && !save) return MODSE_ERR_UNSUPPORTED;
@@ -319,19 +368,28 @@ modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const mo
         tm.mark(3, 1);
         SimtGemmArgs b{p.hm, weights->w_down, p.o, 0};
         MODSE_STAGE(tm, 4, launch_simt_gemm(dtype, kDown, m, L.Pmax, p, b, s, &launches));
+        MODSE_STAGE(tm, 5, launch_combine(dtype, m, n_tokens, L.Pmax, p, y, of32, s, &launches));
     } else {
-        TcMaps maps;
-        if (!tc_fill_maps(maps, m, L, p, weights, false)) return MODSE_ERR_CUDA;
-        MODSE_STAGE(tm, 3, tc_launch(layer->tc, TcUpGate, maps, m, p, nullptr, save, false, s, &launches));
-        MODSE_STAGE(tm, 4, tc_launch(layer->tc, TcDown, maps, m, p, nullptr, save, false, s, &launches));
+        const TcMaps *maps = cached_maps(layer, m, L, p, weights, x, workspace, false);
+        if (maps == nullptr) return MODSE_ERR_CUDA;
+        MODSE_STAGE(tm, 3, tc_launch(layer->tc, TcUpGate, *maps, m, L, p, nullptr, save, false, fuse, nullptr, s, &launches));
+        if (fuse & kFuseScatter) {
+            // y starts at zero and every assignment's gated expert output is added into its token's row
+            MODSE_STAGE(tm, 5, cudaMemsetAsync(y, 0, (size_t)n_tokens * m.d * sizeof(float), s));
+            MODSE_STAGE(tm, 4, tc_launch(layer->tc, TcDown, *maps, m, L, p, nullptr, save, false, fuse,
+                                         static_cast<float *>(y), s, &launches));
+        } else {
+            MODSE_STAGE(tm, 4, tc_launch(layer->tc, TcDown, *maps, m, L, p, nullptr, save, false, fuse, nullptr, s, &launches));
+            MODSE_STAGE(tm, 5, launch_combine(dtype, m, n_tokens, L.Pmax, p, y, of32, s, &launches));
+        }
     }
-    MODSE_STAGE(tm, 5, launch_combine(dtype, m, n_tokens, p, y, of32, s, &launches));
 
     layer->fwd_ws = workspace;
     layer->fwd_tokens = n_tokens;
     layer->fwd_dtype = (int)dtype;
     layer->fwd_saved = save ? 1 : 0;
     layer->fwd_noise = layer->noise.w_noise != nullptr ? 1 : 0;
+    layer->fwd_fuse = fuse;
     layer->last_launches = launches;
     return MODSE_OK;
 }
@@ -360,9 +418,16 @@ modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const m
     int launches = 0;
     const bool of32 = dtype == MODSE_BF16 && layer->out_f32 != 0;
     if (of32 && tc_force_simt()) return MODSE_ERR_UNSUPPORTED;
+    // backward follows the forward it belongs to: a forward that added into y wrote no o, so dg must come from
+    // the row dot; a forward with o may use either
+    const int fuse = (layer->fwd_fuse & kFuseScatter) ? (of32 ? layer->fwd_fuse : -1)
+                                                      : (effective_fuse(layer, dtype, of32) & ~kFuseScatter);
+    if (fuse < 0) return MODSE_ERR_STATE;
 
     StageTimer tm(layer, s);
-    MODSE_STAGE(tm, 6, launch_dg_permute(dtype, m, dy, n_tokens, p, s, &launches));
+    MODSE_CUDA(cudaMemsetAsync(p.status + 4 + TcDownDgrad, 0, 4 * sizeof(int), s));   // tile counters of the backward products
+    MODSE_STAGE(tm, 6, launch_dg_permute(dtype, m, dy, n_tokens, L.Pmax, p, !(fuse & kFuseDgRowdot), s, &launches));
+    bool dx_holds_sum = false;
     if (dtype == MODSE_F32 || tc_force_simt()) {
         SimtGemmArgs a{p.dyp, weights->w_down, p.da, 0};                       // dHm into the dA buffer
         tm.mark(7, 0);
@@ -384,15 +449,24 @@ modse_status_t modse_backward(modse_layer_t *layer, modse_dtype_t dtype, const m
         MODSE_CUDA(launch_simt_gemm(dtype, kUpGateWgrad, m, L.Pmax, p, wg, s, &launches));
         tm.mark(10, 1);
     } else {
-        TcMaps maps;
-        if (!tc_fill_maps(maps, m, L, p, weights, true)) return MODSE_ERR_CUDA;
-        MODSE_STAGE(tm, 7, tc_launch(layer->tc, TcDownDgrad, maps, m, p, wgrads, true, of32, s, &launches));
-        MODSE_STAGE(tm, 8, tc_launch(layer->tc, TcDownWgrad, maps, m, p, wgrads, true, of32, s, &launches));
-        MODSE_STAGE(tm, 9, tc_launch(layer->tc, TcUpGateDgrad, maps, m, p, wgrads, true, of32, s, &launches));
-        MODSE_STAGE(tm, 10, tc_launch(layer->tc, TcUpGateWgrad, maps, m, p, wgrads, true, of32, s, &launches));
+        const TcMaps *maps = cached_maps(layer, m, L, p, weights, x, workspace, true);
+        if (maps == nullptr) return MODSE_ERR_CUDA;
+        MODSE_STAGE(tm, 7, tc_launch(layer->tc, TcDownDgrad, *maps, m, L, p, wgrads, true, of32, fuse, nullptr, s, &launches));
+        MODSE_STAGE(tm, 8, tc_launch(layer->tc, TcDownWgrad, *maps, m, L, p, wgrads, true, of32, fuse, nullptr, s, &launches));
+        if (fuse & kFuseScatter) {
+            tm.mark(9, 0);
+            MODSE_CUDA(cudaMemsetAsync(dx, 0, (size_t)n_tokens * m.d * sizeof(float), s));
+            MODSE_CUDA(tc_launch(layer->tc, TcUpGateDgrad, *maps, m, L, p, wgrads, true, of32, fuse,
+                                 static_cast<float *>(dx), s, &launches));
+            tm.mark(9, 1);
+            dx_holds_sum = true;
+        } else {
+            MODSE_STAGE(tm, 9, tc_launch(layer->tc, TcUpGateDgrad, *maps, m, L, p, wgrads, true, of32, fuse, nullptr, s, &launches));
+        }
+        MODSE_STAGE(tm, 10, tc_launch(layer->tc, TcUpGateWgrad, *maps, m, L, p, wgrads, true, of32, fuse, nullptr, s, &launches));
     }
-    MODSE_STAGE(tm, 11, launch_router_bwd(dtype, m, x, weights->w_router, n_tokens, L.nblk_bwd, p, dx, of32,
-                                          static_cast<float *>(wgrads->dw_router),
+    MODSE_STAGE(tm, 11, launch_router_bwd(dtype, m, x, weights->w_router, n_tokens, L.Pmax, L.nblk_bwd, p, dx, of32,
+                                          dx_holds_sum, static_cast<float *>(wgrads->dw_router),
                                           layer->aux_alpha * (float)m.N / (float)n_tokens, layer->noise, s,
                                           &launches));
     layer->last_launches = launches;
@@ -436,12 +510,48 @@ modse_status_t modse_check_device_status(modse_layer_t *layer, const void *works
 {
     if (layer == nullptr || workspace == nullptr) return MODSE_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    if (layer->debug_checks && layer->fwd_ws == workspace && layer->fwd_tokens > 0) {
+        // compare the guard blocks the last forward wrote; a mismatch lands in the status word
+        const WsLayout L = make_layout(layer->meta, layer->h_desc.data(), layer->fwd_dtype == MODSE_F32 ? 4 : 2,
+                                       layer->fwd_tokens, layer->fwd_saved != 0);
+        void *ws = const_cast<void *>(workspace);
+        if (launch_canaries(ws, L, true, static_cast<int *>(ws), s) != cudaSuccess) return MODSE_ERR_CUDA;
+    }
     int word = 0;
     if (cudaMemcpyAsync(&word, workspace, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return MODSE_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return MODSE_ERR_CUDA;
     if (word == kDevTimeout) return MODSE_ERR_DEVICE_TIMEOUT;
     if (word == kDevBounds) return MODSE_ERR_DEVICE_BOUNDS;
+    return MODSE_OK;
+}
+
+modse_status_t modse_set_debug_checks(modse_layer_t *layer, int on)
+{
+    if (layer == nullptr) return MODSE_ERR_INVALID_ARG;
+    layer->debug_checks = on ? 1 : 0;
+    return MODSE_OK;
+}
+
+modse_status_t modse_set_fusion(modse_layer_t *layer, int flags)
+{
+    if (layer == nullptr || (flags & ~kFuseAll) != 0) return MODSE_ERR_INVALID_ARG;
+    layer->fuse = flags;
+    return MODSE_OK;
+}
+
+int modse_get_fusion(const modse_layer_t *layer) { return layer ? layer->fuse : 0; }
+
+modse_status_t modse_debug_workspace_offsets(const modse_layer_t *layer, modse_dtype_t dtype, int n_tokens,
+                                             int save_for_backward, size_t *prow_of_offset, size_t *first_guard_offset,
+                                             int *padded_rows)
+{
+    if (layer == nullptr || n_tokens < 1 || (dtype != MODSE_F32 && dtype != MODSE_BF16)) return MODSE_ERR_INVALID_ARG;
+    const WsLayout L = make_layout(layer->meta, layer->h_desc.data(), dtype == MODSE_F32 ? 4 : 2, n_tokens,
+                                   save_for_backward != 0);
+    if (prow_of_offset) *prow_of_offset = L.prow_of;
+    if (first_guard_offset) *first_guard_offset = L.canary[1];      // the block behind topk_idx
+    if (padded_rows) *padded_rows = L.Pmax;
     return MODSE_OK;
 }
 
@@ -499,16 +609,16 @@ modse_status_t modse_tune_forward(modse_layer_t *layer, modse_dtype_t dtype, con
     if (cudaEventCreate(&ev[0]) != cudaSuccess) return MODSE_ERR_CUDA;
     if (cudaEventCreate(&ev[1]) != cudaSuccess) { cudaEventDestroy(ev[0]); return MODSE_ERR_CUDA; }
     const int prev = layer->tc.tile_mask;
-    const int base = prev >= 0 ? prev : tc_pair_mask();
-    const int fwd_bits = ((1 << TcUpGate) | (1 << TcDown)) * 0x101;      // both variant bits of the two forward products
-    // candidates: each forward product on the 128-row or on the 256-row kernel.  They are timed in
+    const int base = prev >= 0 ? prev : tc_default_plan();
+    const int fwd_bits = (1 << TcUpGate) | (1 << TcDown);
+    // candidates: each forward product on 128-row or on 256-row tiles.  They are timed in
     // interleaved rounds after a warm-up, so that the drift of the clocks under the power limit (a burst
     // after idle, lower clocks later) does not favour whichever candidate runs first.
     int masks[4];
     float total_ms[4] = {0.f, 0.f, 0.f, 0.f};
     for (int cand = 0; cand < 4; ++cand) {
         const int wide = ((cand & 1) ? (1 << TcUpGate) : 0) | ((cand & 2) ? (1 << TcDown) : 0);
-        masks[cand] = (base & ~fwd_bits) | (wide << 8);
+        masks[cand] = (base & ~fwd_bits) | wide;
     }
     auto run = [&](int reps) {
         for (int rep = 0; rep < reps && st == MODSE_OK; ++rep)
@@ -550,7 +660,7 @@ int modse_get_tile_plan(const modse_layer_t *layer) { return layer ? layer->tc.t
 
 modse_status_t modse_set_tile_plan(modse_layer_t *layer, int plan)
 {
-    if (layer == nullptr || (plan != -1 && (plan < 0 || (plan & ~0x3F3F) != 0))) return MODSE_ERR_INVALID_ARG;
+    if (layer == nullptr || (plan != -1 && (plan < 0 || (plan & ~kTcPlanBits) != 0))) return MODSE_ERR_INVALID_ARG;
     layer->tc.tile_mask = plan;
     return MODSE_OK;
 }
@@ -564,7 +674,13 @@ modse_status_t modse_set_output_f32(modse_layer_t *layer, int on)
 
 void modse_debug_use_fma_path(int on) { tc_set_force_simt(on); }
 
-void modse_debug_set_pair_kernels(int mask) { tc_set_pair_mask(mask); }
+void modse_debug_set_default_tile_plan(int plan) { tc_set_default_plan(plan); }
+
+void modse_debug_set_dynamic_tiles(int on) { tc_set_dynamic_tiles(on); }
+
+void modse_debug_set_wait_limit_ms(int ms) { tc_set_wait_limit_ms(ms); }
+
+void modse_debug_skip_tile_loads(int product, int tile) { tc_set_skip_tile(product, tile); }
 
 const char *modse_stage_name(int stage)
 {

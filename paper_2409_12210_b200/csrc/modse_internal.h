@@ -17,8 +17,14 @@ constexpr int kRouterTokB = 64;     // tokens per block in the router / rank ker
 constexpr int kRouterBwdTokB = 128; // tokens per block in the router backward kernel
 constexpr int kPanel = 64;          // hidden-axis panel width of the bf16 activation layout
 
-// Device status word values (first int of the workspace).
+// Device status word values (first int of the workspace).  Ints 4..9 of the same 64-byte block are the
+// tile counters of the six grouped products (zeroed with it).
 enum : int { kDevOk = 0, kDevTimeout = 1, kDevBounds = 2 };
+
+// Every workspace region is followed by a 256-byte guard block.  With the debug checks on its first 8 bytes
+// hold a pattern derived from the block's index; a kernel that wrote past its region destroys it.
+constexpr int kMaxCanaries = 48;
+constexpr unsigned long long kCanaryPattern = 0x5EDC0DE5CA9A51E5ull;
 
 // Layer shape, passed by value to kernels (prefix sums of the hidden widths).
 struct LayerMeta {
@@ -32,7 +38,10 @@ struct WsLayout {
     size_t hb;   // element capacity of each [padded rows x h_e] activation buffer
     size_t status, topk_idx, topk_gate, counts, counts_slot, offsets, poffsets, ebase, row_of, token_of,
         prow_of, ptoken_of, pgate, block_counts, logits, aux_partial, noise_u, du, dgamma_partial, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
-        total;
+        dg_part, total;
+    int dg_slots;                    // partial row dots per padded row (two per 256-column tile of the widest expert)
+    int n_canary;
+    size_t canary[kMaxCanaries];     // byte offsets of the guard blocks
 };
 
 // Pointers carved out of the workspace (device addresses).
@@ -50,6 +59,7 @@ struct WsPtrs {
     float *du;           // [T,N] gradient w.r.t. x W_n
     float *dgamma_partial;  // [nblk_bwd]
     float *dg, *dz, *dwr_partial;
+    float *dg_part;      // [dg_slots][Pmax] partial sums of dg from the down-dgrad epilogue (fused variant)
     // xp: x in padded expert-grouped rows.  a_pre / b_pre: what the forward keeps for the SwiGLU backward -
     // the pre-activations A = xp W_gate^T, B = xp W_up^T on the fp32 path, B silu'(A) and silu(A) on the bf16
     // path.  hm: gated hidden rows g silu(A) B.  o / dxp: fp32 gated expert outputs / input gradients per row.
@@ -73,16 +83,22 @@ WsPtrs carve(void *ws, const WsLayout &L);
 cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
                           const WsPtrs &p, const NoiseGate &ng, cudaStream_t s, int *launches);
 cudaError_t launch_rank(const LayerMeta &m, int T, int Pmax, const WsPtrs &p, cudaStream_t s, int *launches);
-cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, const WsPtrs &p,
+// Every kernel that follows an index read from the routing tables checks it against Pmax (padded rows) or T
+// (tokens) first; an index outside records kDevBounds in the status word and the access is skipped.
+cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, int Pmax, const WsPtrs &p,
                            cudaStream_t s, int *launches);
-cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, bool out_f32,
+cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, int Pmax, const WsPtrs &p, void *y, bool out_f32,
                            cudaStream_t s, int *launches);
-cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, const WsPtrs &p,
-                              cudaStream_t s, int *launches);
-// aux_scale = alpha * N / T of the auxiliary load-balance loss (Eq. 7), 0 when it is not part of the objective
+// with_dg: also dg[t,j] = <dY_t, o_row> / g from the stored fp32 expert outputs (otherwise only the permutation of dY)
+cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, int Pmax, const WsPtrs &p,
+                              bool with_dg, cudaStream_t s, int *launches);
+// aux_scale = alpha * N / T of the auxiliary load-balance loss (Eq. 7), 0 when it is not part of the objective.
+// dx_holds_sum: dx (fp32) already holds the sum of the token's dxp rows (scatter-adding up/gate dgrad).
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
-                              int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
-                              float aux_scale, const NoiseGate &ng, cudaStream_t s, int *launches);
+                              int Pmax, int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, bool dx_holds_sum,
+                              float *dw_router, float aux_scale, const NoiseGate &ng, cudaStream_t s, int *launches);
+// guard blocks of the workspace: write the patterns / compare them (a mismatch records kDevBounds)
+cudaError_t launch_canaries(void *ws, const WsLayout &L, bool check, int *status, cudaStream_t s);
 // L_a = alpha N sum_i f_i P_i (Eq. 7-10) from the stored logits and the slot-0 histogram
 cudaError_t launch_aux_loss(const LayerMeta &m, int T, int nblk_bwd, const WsPtrs &p, float alpha, float *loss,
                             float *f, float *P, cudaStream_t s, int *launches);

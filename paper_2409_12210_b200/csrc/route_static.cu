@@ -18,8 +18,12 @@ namespace {
 constexpr size_t kStaticScratchBytes = 4u << 20;   // 4 MiB
 static __device__ __align__(256) unsigned char g_route_scratch[kStaticScratchBytes];
 
+// Device address of g_route_scratch per device (host copy).  Valid for this process and the device's
+// current context: it is looked up on the first call, so first calls from several host threads must
+// be serialised by the caller, and a cudaDeviceReset invalidates it (the library is not usable
+// across a reset).
 constexpr int kMaxDevices = 64;
-unsigned char *g_scratch_ptr[kMaxDevices];         // device address of g_route_scratch per device (host copy)
+unsigned char *g_scratch_ptr[kMaxDevices];
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -114,3 +118,20 @@ extern "C" modse_status_t modse_route_static_scratch(modse_dtype_t dtype, int d_
 }
 
 extern "C" size_t modse_route_static_scratch_capacity(void) { return kStaticScratchBytes; }
+
+// The status word of the last modse_route_static_scratch call on the current device lives in the
+// fixed array, where modse_check_device_status (which takes a workspace) cannot reach it.
+extern "C" modse_status_t modse_route_static_scratch_status(void *cuda_stream)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MODSE_ERR_CUDA;
+    if (g_scratch_ptr[dev] == nullptr) return MODSE_OK;          // no call has run on this device yet
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    int word = 0;
+    if (cudaMemcpyAsync(&word, g_scratch_ptr[dev], sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return MODSE_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return MODSE_ERR_CUDA;
+    if (word == modse::kDevTimeout) return MODSE_ERR_DEVICE_TIMEOUT;
+    if (word == modse::kDevBounds) return MODSE_ERR_DEVICE_BOUNDS;
+    return MODSE_OK;
+}

@@ -530,7 +530,8 @@ rank_kernel(LayerMeta m, int Ttok, int Pmax, int nblk, const int *__restrict__ b
 template <typename T>
 __global__ void __launch_bounds__(256)
 permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int *__restrict__ prow_of,
-               const int *__restrict__ counts, const int *__restrict__ poffsets, T *__restrict__ xp, int tok_blocks)
+               const int *__restrict__ counts, const int *__restrict__ poffsets, T *__restrict__ xp, int tok_blocks,
+               int Pmax, int *status)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if ((int)blockIdx.x < tok_blocks) {
@@ -540,6 +541,11 @@ permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int
         int rows[2];
         rows[0] = prow_of[(size_t)t * k];
         rows[1] = (k > 1) ? prow_of[(size_t)t * k + 1] : -1;
+        for (int j = 0; j < k; ++j)
+            if (rows[j] < 0 || rows[j] >= Pmax) {            // a row outside the padded group space: skipped
+                if (lane == 0) atomicMax(status, kDevBounds);
+                rows[j] = -1;
+            }
         for (int c = lane * 8; c < d; c += 256) {
             float v[8];
             load8(src + c, v);
@@ -554,6 +560,7 @@ permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int
         if (e >= N) return;
         const int row = poffsets[e] + counts[e] + i;
         if (row >= poffsets[e + 1]) return;
+        if (row < 0 || row >= Pmax) { if (lane == 0) atomicMax(status, kDevBounds); return; }
         const float zero[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int c = lane * 8; c < d; c += 256) store8(xp + (size_t)row * d + c, zero);
     }
@@ -567,13 +574,17 @@ permute_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const int
 template <typename TO>
 __global__ void __launch_bounds__(256)
 combine_kernel(const float *__restrict__ o, int Ttok, int d, int k, const int *__restrict__ prow_of,
-               TO *__restrict__ y)
+               TO *__restrict__ y, int Pmax, int *status)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * 8 + warp;
     if (t >= Ttok) return;
     const int r0 = prow_of[(size_t)t * k];
     const int r1 = (k > 1) ? prow_of[(size_t)t * k + 1] : -1;
+    if (r0 < 0 || r0 >= Pmax || r1 >= Pmax || (k > 1 && r1 < 0)) {
+        if (lane == 0) atomicMax(status, kDevBounds);
+        return;
+    }
     for (int c = lane * 8; c < d; c += 256) {
         float a[8], acc[8];
         load8(o + (size_t)r0 * d + c, acc);
@@ -591,32 +602,55 @@ combine_kernel(const float *__restrict__ o, int Ttok, int d, int k, const int *_
 // the gated expert output; a gate that underflowed to 0 gives dg = 0, and its
 // dz = g*(dg - s) is 0 either way); dyp[row(t,j)] = dY_t, an exact copy.
 // ---------------------------------------------------------------------------
-template <typename T>
+// WITH_DG = false: only the permutation of dY (dg then comes from the down-dgrad epilogue).
+template <typename T, bool WITH_DG>
 __global__ void __launch_bounds__(256)
 dg_permute_kernel(const T *__restrict__ dy, const float *__restrict__ o, int Ttok, int d, int N, int k,
                   const int *__restrict__ prow_of, const float *__restrict__ topk_gate,
                   const int *__restrict__ counts, const int *__restrict__ poffsets, float *__restrict__ dg,
-                  T *__restrict__ dyp, int tok_blocks)
+                  T *__restrict__ dyp, int tok_blocks, int Pmax, int *status)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if ((int)blockIdx.x < tok_blocks) {
         const int t = blockIdx.x * 8 + warp;
         if (t >= Ttok) return;
         const T *src = dy + (size_t)t * d;
-        for (int j = 0; j < k; ++j) {
-            const int row = prow_of[(size_t)t * k + j];
-            const float g = topk_gate[(size_t)t * k + j];
-            float acc = 0.f;
-            for (int c = lane * 8; c < d; c += 256) {
-                float v[8], ov[8];
-                load8(src + c, v);
-                load8(o + (size_t)row * d + c, ov);
+        if constexpr (WITH_DG) {
+            for (int j = 0; j < k; ++j) {
+                const int row = prow_of[(size_t)t * k + j];
+                if (row < 0 || row >= Pmax) {
+                    if (lane == 0) { atomicMax(status, kDevBounds); dg[(size_t)t * k + j] = 0.f; }
+                    continue;
+                }
+                const float g = topk_gate[(size_t)t * k + j];
+                float acc = 0.f;
+                for (int c = lane * 8; c < d; c += 256) {
+                    float v[8], ov[8];
+                    load8(src + c, v);
+                    load8(o + (size_t)row * d + c, ov);
 #pragma unroll
-                for (int u = 0; u < 8; ++u) acc = fmaf(v[u], ov[u], acc);
-                store8(dyp + (size_t)row * d + c, v);
+                    for (int u = 0; u < 8; ++u) acc = fmaf(v[u], ov[u], acc);
+                    store8(dyp + (size_t)row * d + c, v);
+                }
+                acc = warp_sum(acc);
+                if (lane == 0) dg[(size_t)t * k + j] = (g > 0.f) ? acc / g : 0.f;
             }
-            acc = warp_sum(acc);
-            if (lane == 0) dg[(size_t)t * k + j] = (g > 0.f) ? acc / g : 0.f;
+        } else {
+            int rows[2];
+            rows[0] = prow_of[(size_t)t * k];
+            rows[1] = (k > 1) ? prow_of[(size_t)t * k + 1] : -1;
+            for (int j = 0; j < k; ++j)
+                if (rows[j] < 0 || rows[j] >= Pmax) {
+                    if (lane == 0) atomicMax(status, kDevBounds);
+                    rows[j] = -1;
+                }
+            for (int c = lane * 8; c < d; c += 256) {
+                float v[8];
+                load8(src + c, v);
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+                    if (rows[j] >= 0) store8(dyp + (size_t)rows[j] * d + c, v);
+            }
         }
     } else {
         const int pb = blockIdx.x - tok_blocks;
@@ -624,6 +658,7 @@ dg_permute_kernel(const T *__restrict__ dy, const float *__restrict__ o, int Tto
         if (e >= N) return;
         const int row = poffsets[e] + counts[e] + i;
         if (row >= poffsets[e + 1]) return;
+        if (row < 0 || row >= Pmax) { if (lane == 0) atomicMax(status, kDevBounds); return; }
         const float zero[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
         for (int c = lane * 8; c < d; c += 256) store8(dyp + (size_t)row * d + c, zero);
     }
@@ -788,7 +823,8 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
                  const int *__restrict__ topk_idx, const float *__restrict__ topk_gate,
                  const int *__restrict__ prow_of, const float *__restrict__ dg, float *__restrict__ dz,
                  TO *__restrict__ dx, int N, const float *__restrict__ logits, const int *__restrict__ counts_slot,
-                 float aux_scale, const T *__restrict__ w_noise, const float *__restrict__ du)
+                 float aux_scale, const T *__restrict__ w_noise, const float *__restrict__ du, int Pmax,
+                 int dx_holds_sum, int *status)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * 8 + warp;
@@ -800,6 +836,10 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
         dgv[j] = dg[(size_t)t * k + j];
         e[j] = topk_idx[(size_t)t * k + j];
         rows[j] = prow_of[(size_t)t * k + j];
+        if (rows[j] < 0 || rows[j] >= Pmax || e[j] < 0 || e[j] >= N) {   // skipped: the token's dx row is left unwritten
+            if (lane == 0) atomicMax(status, kDevBounds);
+            return;
+        }
     }
     const float s = g[0] * dgv[0] + g[1] * dgv[1];
     dzv[0] = g[0] * (dgv[0] - s);
@@ -812,11 +852,21 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
     if (aux_scale != 0.f) token_softmax_stats(zt, counts_slot, N, inv_T, zmax, inv_den, fp);
     for (int c = lane * 8; c < d; c += 256) {
         float a[8], out[8], wv[8];
-        load8(dxp + (size_t)rows[0] * d + c, out);
-        if (k > 1) {
-            load8(dxp + (size_t)rows[1] * d + c, a);
+        if (dx_holds_sum) {
+            // the up/gate dgrad added the token's rows into dx (fp32) already
+            if constexpr (sizeof(TO) == 4) {
+                load8(reinterpret_cast<const float *>(dx) + (size_t)t * d + c, out);
+            } else {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) out[u] += a[u];
+                for (int u = 0; u < 8; ++u) out[u] = 0.f;      // not reached: adding into dx needs fp32 outputs
+            }
+        } else {
+            load8(dxp + (size_t)rows[0] * d + c, out);
+            if (k > 1) {
+                load8(dxp + (size_t)rows[1] * d + c, a);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) out[u] += a[u];
+            }
         }
         for (int j = 0; j < k; ++j) {
             load8(w_router + (size_t)e[j] * d + c, wv);
@@ -1004,56 +1054,91 @@ cudaError_t launch_rank(const LayerMeta &m, int T, int Pmax, const WsPtrs &p, cu
     return cudaSuccess;
 }
 
-cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, const WsPtrs &p,
+cudaError_t launch_permute(modse_dtype_t dt, const LayerMeta &m, const void *x, int T, int Pmax, const WsPtrs &p,
                            cudaStream_t s, int *launches)
 {
     const int tok_blocks = (T + 7) / 8;
     const int grid = tok_blocks + m.N * 16;
     if (dt == MODSE_F32)
         permute_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.prow_of, p.counts,
-                                                   p.poffsets, (float *)p.xp, tok_blocks);
+                                                   p.poffsets, (float *)p.xp, tok_blocks, Pmax, p.status);
     else
         permute_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k, p.prow_of,
-                                                           p.counts, p.poffsets, (__nv_bfloat16 *)p.xp, tok_blocks);
+                                                           p.counts, p.poffsets, (__nv_bfloat16 *)p.xp, tok_blocks,
+                                                           Pmax, p.status);
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
 }
 
-cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, const WsPtrs &p, void *y, bool out_f32,
+cudaError_t launch_combine(modse_dtype_t dt, const LayerMeta &m, int T, int Pmax, const WsPtrs &p, void *y, bool out_f32,
                            cudaStream_t s, int *launches)
 {
     const int grid = (T + 7) / 8;
     if (dt == MODSE_F32 || out_f32)
-        combine_kernel<float><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of, (float *)y);
+        combine_kernel<float><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of, (float *)y, Pmax,
+                                                   p.status);
     else
         combine_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const float *)p.o, T, m.d, m.k, p.prow_of,
-                                                           (__nv_bfloat16 *)y);
+                                                           (__nv_bfloat16 *)y, Pmax, p.status);
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
 }
 
-cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, const WsPtrs &p,
-                              cudaStream_t s, int *launches)
+template <typename T, bool WITH_DG>
+static void launch_dg_permute_t(const LayerMeta &m, const void *dy, int Ttok, int Pmax, const WsPtrs &p, cudaStream_t s)
 {
-    const int tok_blocks = (T + 7) / 8;
+    const int tok_blocks = (Ttok + 7) / 8;
     const int grid = tok_blocks + m.N * 16;
-    if (dt == MODSE_F32)
-        dg_permute_kernel<float><<<grid, 256, 0, s>>>((const float *)dy, (const float *)p.o, T, m.d, m.N, m.k,
-                                                      p.prow_of, p.topk_gate, p.counts, p.poffsets, p.dg,
-                                                      (float *)p.dyp, tok_blocks);
-    else
-        dg_permute_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)dy,
-                                                              (const float *)p.o, T, m.d, m.N, m.k,
-                                                              p.prow_of, p.topk_gate, p.counts, p.poffsets, p.dg,
-                                                              (__nv_bfloat16 *)p.dyp, tok_blocks);
+    dg_permute_kernel<T, WITH_DG><<<grid, 256, 0, s>>>((const T *)dy, (const float *)p.o, Ttok, m.d, m.N, m.k, p.prow_of,
+                                                       p.topk_gate, p.counts, p.poffsets, p.dg, (T *)p.dyp, tok_blocks,
+                                                       Pmax, p.status);
+}
+
+cudaError_t launch_dg_permute(modse_dtype_t dt, const LayerMeta &m, const void *dy, int T, int Pmax, const WsPtrs &p,
+                              bool with_dg, cudaStream_t s, int *launches)
+{
+    if (dt == MODSE_F32) {
+        if (with_dg) launch_dg_permute_t<float, true>(m, dy, T, Pmax, p, s);
+        else launch_dg_permute_t<float, false>(m, dy, T, Pmax, p, s);
+    } else {
+        if (with_dg) launch_dg_permute_t<__nv_bfloat16, true>(m, dy, T, Pmax, p, s);
+        else launch_dg_permute_t<__nv_bfloat16, false>(m, dy, T, Pmax, p, s);
+    }
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
+}
+
+// Guard blocks between the workspace regions: block i holds kCanaryPattern ^ i in its first 8 bytes.
+struct CanaryOffsets {
+    int n;
+    size_t off[kMaxCanaries];
+};
+namespace {
+__global__ void canary_kernel(unsigned char *ws, CanaryOffsets c, int check, int *status)
+{
+    const int i = threadIdx.x;
+    if (i >= c.n) return;
+    unsigned long long *w = reinterpret_cast<unsigned long long *>(ws + c.off[i]);
+    const unsigned long long want = kCanaryPattern ^ (unsigned long long)i;
+    if (!check) *w = want;
+    else if (*w != want) atomicMax(status, kDevBounds);
+}
+}  // namespace
+
+cudaError_t launch_canaries(void *ws, const WsLayout &L, bool check, int *status, cudaStream_t s)
+{
+    CanaryOffsets c;
+    c.n = L.n_canary;
+    for (int i = 0; i < kMaxCanaries; ++i) c.off[i] = i < L.n_canary ? L.canary[i] : 0;
+    canary_kernel<<<1, 64, 0, s>>>(static_cast<unsigned char *>(ws), c, check ? 1 : 0, status);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *x, const void *w_router, int T,
-                              int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, float *dw_router,
-                              float aux_scale, const NoiseGate &ng, cudaStream_t s, int *launches)
+                              int Pmax, int nblk_bwd, const WsPtrs &p, void *dx, bool out_f32, bool dx_holds_sum,
+                              float *dw_router, float aux_scale, const NoiseGate &ng, cudaStream_t s, int *launches)
 {
+    const int hs = dx_holds_sum ? 1 : 0;
     const bool noise = ng.w_noise != nullptr;
     const float *du = noise ? p.du : nullptr;
     if (noise) {
@@ -1069,16 +1154,19 @@ cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *
     if (dt == MODSE_F32)
         router_dx_kernel<float, float><<<grid_dx, 256, 0, s>>>((const float *)w_router, dxp, T, m.d, m.k, p.topk_idx,
                                                                p.topk_gate, p.prow_of, p.dg, p.dz, (float *)dx, m.N, p.logits,
-                                                               p.counts_slot, aux_scale, (const float *)ng.w_noise, du);
+                                                               p.counts_slot, aux_scale, (const float *)ng.w_noise, du,
+                                                               Pmax, hs, p.status);
     else if (out_f32)
         router_dx_kernel<__nv_bfloat16, float><<<grid_dx, 256, 0, s>>>((const __nv_bfloat16 *)w_router, dxp, T, m.d,
                                                                        m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg,
                                                                        p.dz, (float *)dx, m.N, p.logits, p.counts_slot,
-                                                                       aux_scale, (const __nv_bfloat16 *)ng.w_noise, du);
+                                                                       aux_scale, (const __nv_bfloat16 *)ng.w_noise, du,
+                                                                       Pmax, hs, p.status);
     else
         router_dx_kernel<__nv_bfloat16, __nv_bfloat16><<<grid_dx, 256, 0, s>>>(
             (const __nv_bfloat16 *)w_router, dxp, T, m.d, m.k, p.topk_idx, p.topk_gate, p.prow_of, p.dg, p.dz,
-            (__nv_bfloat16 *)dx, m.N, p.logits, p.counts_slot, aux_scale, (const __nv_bfloat16 *)ng.w_noise, du);
+            (__nv_bfloat16 *)dx, m.N, p.logits, p.counts_slot, aux_scale, (const __nv_bfloat16 *)ng.w_noise, du, Pmax, hs,
+            p.status);
     MODSE_LAUNCH_CHECK();
     dim3 grid(nblk_bwd, dt == MODSE_F32 ? (m.d + 255) / 256 : (m.d + 511) / 512);
     const int n = m.N * m.d;

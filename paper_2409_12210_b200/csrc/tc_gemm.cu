@@ -1,8 +1,8 @@
 // Grouped GEMMs of the bf16 MoDSE layer on Blackwell tensor cores.
 //
 // One persistent, warp-specialised kernel template serves the six products of
-// the layer (Sec. 3.1, Eq. 4 and its gradient); a tile is 128 rows by up to 256
-// fp32 accumulator columns held in tensor memory (TMEM):
+// the layer (Sec. 3.1, Eq. 4 and its gradient); the accumulators (fp32) live in
+// tensor memory (TMEM):
 //
 //   kind            product (per expert e, cp = padded rows, h = width)      K
 //   UpGate          Hm = g * silu(xp Wg^T) * (xp Wu^T)      [cp, h]          d
@@ -12,15 +12,18 @@
 //   UpGateDgrad     dxp = dA Wg_e + dB Wu_e                 [cp, d]  fp32    2h
 //   UpGateWgrad     dWg_e = dA^T xp, dWu_e = dB^T xp        [h, d]           cp
 //
-// Roles inside a CTA (320 threads): warp 0 issues TMA loads into a 4-stage
-// shared-memory ring (every box is 64 elements x 64 rows, 128-byte swizzle),
-// warp 1 issues tcgen05.mma with the accumulator in TMEM (two accumulators, so
-// the epilogue of one tile overlaps the main loop of the next), warps 2-9 read
+// Two tile shapes: 128 rows x up to 256 accumulator columns with two
+// accumulators in flight (the epilogue of one tile overlaps the main loop of the
+// next), and 256 rows (two 128-row halves that share the column operand, 2/3 of
+// the shared-memory traffic per FLOP, but both accumulators belong to one tile).
+//
+// Roles inside a CTA (352 threads): warp 0 issues TMA loads into a ring of
+// shared-memory stages (boxes of 64 elements x 64 or 128 rows, 128-byte
+// swizzle), warp 1 issues tcgen05.mma, warp 2 hands out tiles, warps 3-10 read
 // the accumulator with tcgen05.ld (two warps per TMEM lane quadrant, each half
-// of the columns) and run the fused epilogue.  Operands are
-// consumed either K-major or MN-major straight from their row-major buffers
-// (the instruction descriptor carries the major-ness), so the backward pass
-// needs no transposed copies.
+// of the tile's columns) and run the fused epilogue.  Operands are consumed either K-major or MN-major
+// straight from their row-major buffers (the instruction descriptor carries the
+// major-ness), so the backward pass needs no transposed copies.
 //
 // (g = gate of the row's assignment: it is applied to the hidden row, in fp32,
 // before the one rounding to bf16, so neither o nor dY needs a rounded gated
@@ -31,16 +34,25 @@
 // rounded factor each instead of two rounded pre-activations.
 //
 // Activations that have the hidden axis as their width (Hm, sp, sq, dA, dB)
-// are stored as panels: for expert e, panel pc holds
-// columns [64 pc, 64 pc + 64) of all cp rows contiguously, so that a single
-// two-dimensional tensor map with 128-byte rows describes the whole buffer
-// although the row length h differs from expert to expert.
+// are stored as panels: for expert e, panel pc holds columns [64 pc, 64 pc + 64)
+// of all cp rows contiguously, so that a single two-dimensional tensor map with
+// 128-byte rows describes the whole buffer although the row length h differs
+// from expert to expert.
 //
-// Tiles are handed out statically: experts are ordered by decreasing K so the
-// long tiles of wide experts (or of experts with many tokens) start first and
-// the short ones fill the tail - the one-GPU form of the paper's expert-pair
-// balancing (Sec. 3.2).  Every wait is bounded; a wait that expires records
-// kDevTimeout in the status word and the CTA drains and exits.
+// Tile order: experts by decreasing K, so the long tiles of wide experts (or of
+// experts with many tokens) start first and the short ones fill the tail - the
+// one-GPU form of the paper's expert-pair balancing (Sec. 3.2).  CTAs take the
+// next tile of that list from a counter in global memory (or, with the
+// counter switched off, are dealt tiles round-robin).  Every output tile is
+// computed by one CTA with its K blocks in ascending order either way, so the
+// results do not depend on which CTA ran which tile.  The counter is read by a
+// warp of its own, which passes the tile indices to the three working roles
+// through a small queue in shared memory: an atomic instruction inside the
+// loop of the thread that issues the TMA loads cost the 128-row kernels a
+// quarter of their speed (measured, even with the instruction never executed).
+//
+// Every wait is bounded; a wait that expires records kDevTimeout in the status
+// word and the CTA drains and exits.
 #include <cuda.h>
 
 #include "tc_gemm.h"
@@ -48,57 +60,78 @@
 namespace modse {
 
 static int g_force_simt = 0;
-static int g_pair_mask = 0;      // bit k: product kind k runs on the two-CTA kernel
-// bit k: product kind k runs on the 256-row single-CTA kernel.  Default: the four products with long
-// K loops (down, down wgrad, up/gate dgrad, up/gate wgrad), where it measured 4-13 % faster than the
-// 128-row kernel; the two products with K = d and heavy epilogues (up/gate, down dgrad) measured slower.
-static int g_wide_mask = (1 << 1) | (1 << 3) | (1 << 4) | (1 << 5);
-void tc_set_pair_mask(int mask) { g_pair_mask = mask & 63; g_wide_mask = (mask >> 8) & 63; }
-int tc_pair_mask() { return g_pair_mask | (g_wide_mask << 8); }
+static int g_default_plan = kTcDefaultPlan;
+static int g_dynamic_tiles = 1;
+static int g_wait_limit_ms = 2000;
+static int g_skip_kind = -1, g_skip_tile = -1;
 
 bool tc_force_simt() { return g_force_simt != 0; }
 void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
+void tc_set_default_plan(int mask) { g_default_plan = mask & kTcPlanBits; }
+int tc_default_plan() { return g_default_plan; }
+void tc_set_dynamic_tiles(int on) { g_dynamic_tiles = on ? 1 : 0; }
+void tc_set_wait_limit_ms(int ms) { g_wait_limit_ms = ms < 1 ? 1 : (ms > 60000 ? 60000 : ms); }
+void tc_set_skip_tile(int kind, int tile) { g_skip_kind = kind; g_skip_tile = tile; }
 
 namespace {
 
-constexpr int kStages = 4;
 constexpr int kBoxBytes = 64 * 64 * 2;           // one TMA box: 64 rows of 128 bytes
 constexpr int kARegion = 2 * kBoxBytes;          // 128 rows (or 128 MN elements) x 64 K
 constexpr int kBRegion = 4 * kBoxBytes;          // up to 256 rows x 64 K
-constexpr int kStageBytes = kARegion + kBRegion; // 48 KB
-constexpr int kThreads = 320;                   // TMA warp, MMA warp, eight epilogue warps
+constexpr int kEpiWarps = 8;
+constexpr int kFirstEpiWarp = 3;
+constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);   // TMA warp, MMA warp, tile warp, eight epilogue warps
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s per wait
 constexpr int kEpiRowBytes = 64;                 // a 32-element bf16 chunk of one row; 16-byte pieces XOR-swizzled
-constexpr int kEpiWarpBytes = 32 * kEpiRowBytes;
+constexpr int kEpiBufBytes = 32 * kEpiRowBytes;  // one warp's 32 rows: 2 KB
+constexpr int kEpiBytes = kEpiWarps * kEpiBufBytes;   // one transposing buffer per epilogue warp
+constexpr int kTileQ = 4;                        // tile indices in flight between the producer and the other roles
+
+// 128-row tiles: 4 stages of 16 KB rows + 32 KB columns.  256-row tiles: 3 stages of 2 x 16 KB rows + 32 KB columns.
+template <bool WIDE> struct Shape {
+    static constexpr int kStages = WIDE ? 3 : 4;
+    static constexpr int kRowRegion = WIDE ? 2 * kARegion : kARegion;
+    static constexpr int kStageBytes = kRowRegion + kBRegion;
+    static constexpr int kTileRows = WIDE ? 256 : 128;
+};
 
 struct TcParams {
     LayerMeta meta;
     const int *poffsets;
     const long long *ebase;
     int *status;
+    int *tile_counter;            // this product's counter of tiles handed out (zero at launch)
     const float *pgate;           // gate of the assignment in each padded row (0 for padding)
+    const int *ptoken_of;         // token of each padded row (-1 for padding)
     __nv_bfloat16 *hm, *da, *db;
     __nv_bfloat16 *sp, *sq;       // saved for backward: sp = B * silu'(A), sq = silu(A) (panel layout)
     float *o, *dxp;
     __nv_bfloat16 *dw_gate, *dw_up, *dw_down;
+    float *dg_part;               // [slots][Pmax] partial row dots of the down dgrad with Hm
+    float *scatter_out;           // fp32 [T, d] target of the scatter-adding epilogues
+    unsigned long long wait_limit_ns;
+    int Pmax, T;
     int save;
     int out_f32;   // weight gradients are written as fp32 instead of bf16
+    int dynamic;   // tiles come from the global counter
+    int skip_tile; // debugging: the producer that gets this tile stops without loading it (-1: none)
 };
 
-// dynamic shared memory map (after 1024-byte alignment)
+// control block behind the stages and the epilogue buffers
 struct SmemTail {
-    unsigned char epi_stage[8][kEpiWarpBytes];   // one transposing buffer per epilogue warp
-    unsigned long long full[kStages], empty[kStages], tmem_full[2], tmem_empty[2];
+    unsigned long long full[4], empty[4], tmem_full[2], tmem_empty[2], tq_full[kTileQ], tq_empty[kTileQ], tq_taken;
     unsigned int tmem_base;
     int abort_flag;
-    int order[kMaxExperts];
-    int key[kMaxExperts];
-    int ntile[kMaxExperts];
+    int tile_q[kTileQ];
     int tstart[kMaxExperts + 1];
+    unsigned short order[kMaxExperts];
 };
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(SmemTail);
+template <bool WIDE> constexpr size_t smem_bytes()
+{
+    return 1024 + (size_t)Shape<WIDE>::kStages * Shape<WIDE>::kStageBytes + kEpiBytes + sizeof(SmemTail);
+}
+static_assert(smem_bytes<false>() <= 232448 && smem_bytes<true>() <= 232448, "shared memory per CTA");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -132,17 +165,24 @@ __device__ __forceinline__ unsigned long long global_ns()
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: false if the phase did not complete within kWaitLimitNs or the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *status)
+
+// What a role needs to give up a wait: the CTA's abort flag, the status word and the time limit.
+struct WaitCtx {
+    volatile int *abort_flag;
+    int *status;
+    unsigned long long limit_ns;
+};
+// Bounded wait: false if the phase did not complete within the limit or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx &w)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     unsigned it = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++it & 255u) == 0) {
-            if (*abort_flag || global_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicMax(status, kDevTimeout);
+            if (*w.abort_flag || global_ns() - t0 > w.limit_ns) {
+                *w.abort_flag = 1;
+                atomicMax(w.status, kDevTimeout);
                 return false;
             }
         }
@@ -157,7 +197,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
-
+// Four rows y0..y3 of a tensor whose map has boxes one row high, into four consecutive 128-byte rows at dst
+// (a row index outside the tensor reads zeros).
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y0, int y1,
+                                            int y2, int y3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y0), "r"(y1), "r"(y2), "r"(y3)
+        : "memory");
+}
 // `nboxes` 64-row boxes stacked from row y on (K-major operand): pairs of them go as one 128-row copy.
 __device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap *m64, const CUtensorMap *m128, uint32_t bar,
                                               int x, int y, int nboxes)
@@ -217,12 +267,11 @@ __device__ __forceinline__ uint32_t make_idesc(bool a_mn, bool b_mn, int n)
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
-// Tiles are dealt to the CTAs in rounds of one tile each.  The tile list is sorted by decreasing length of
-// the K loop, so within a round the first CTA gets the longest tile; where K is the expert's width (down,
-// up/gate dgrad) dealing every round in the same direction hands the same CTAs the longer tile of every
-// round (12 % above the mean load for the benchmark's widths), so odd rounds run through the CTAs in
-// reverse order, which evens that out (5.5 %, as good as dealing each tile to the least loaded CTA).
-// Measured: 4 % on those two products.
+// Static hand-out (the global counter switched off): tiles are dealt to the CTAs in rounds of one tile each.
+// The tile list is sorted by decreasing length of the K loop, so within a round the first CTA gets the
+// longest tile; where K is the expert's width (down, up/gate dgrad) dealing every round in the same
+// direction hands the same CTAs the longer tile of every round (12 % above the mean load for the
+// benchmark's widths), so odd rounds run through the CTAs in reverse order, which evens that out (5.5 %).
 template <int KIND>
 __device__ __forceinline__ int dealt_tile(int round, int who, int n)
 {
@@ -281,22 +330,25 @@ struct Tile {
     int e, cp, h, ho, prow0, pbase;   // expert, padded rows, width, width offset, first padded row, first panel row
     int m0, n0, mrows, ncols, nk, which;
     int n_mma, a_boxes, b_boxes;
-    int a_boxes_peer, b_off;          // two-CTA tiles only: boxes of the partner's rows, this CTA's column offset
+    int a_boxes_peer;                 // 256-row tiles: boxes of the second 128-row half
 };
 
 // tiles (rows, columns) and K blocks of one expert
-template <int KIND>
+template <int KIND, bool WIDE>
 __device__ __forceinline__ void expert_shape(int cp, int h, int d, int &mt, int &nt, int &nk)
 {
-    if constexpr (KIND == TcUpGate)      { mt = cp / 128; nt = (h + 127) / 128; nk = d / 64; }
-    if constexpr (KIND == TcDown)        { mt = cp / 128; nt = (d + 255) / 256; nk = h / 64; }
-    if constexpr (KIND == TcDownDgrad)   { mt = cp / 128; nt = (h + 255) / 256; nk = d / 64; }
-    if constexpr (KIND == TcDownWgrad)   { mt = d / 128;  nt = (h + 255) / 256; nk = cp / 64; }
-    if constexpr (KIND == TcUpGateDgrad) { mt = cp / 128; nt = (d + 255) / 256; nk = 2 * (h / 64); }
-    if constexpr (KIND == TcUpGateWgrad) { mt = 2 * ((h + 127) / 128); nt = (d + 255) / 256; nk = cp / 64; }
+    constexpr int R = WIDE ? 256 : 128;
+    if constexpr (KIND == TcUpGate)      { mt = (cp + R - 1) / R; nt = (h + 127) / 128; nk = d / 64; }
+    if constexpr (KIND == TcDown)        { mt = (cp + R - 1) / R; nt = (d + 255) / 256; nk = h / 64; }
+    if constexpr (KIND == TcDownDgrad)   { mt = (cp + R - 1) / R; nt = (h + 255) / 256; nk = d / 64; }
+    if constexpr (KIND == TcDownWgrad)   { mt = (d + R - 1) / R;  nt = (h + 255) / 256; nk = cp / 64; }
+    if constexpr (KIND == TcUpGateDgrad) { mt = (cp + R - 1) / R; nt = (d + 255) / 256; nk = 2 * (h / 64); }
+    if constexpr (KIND == TcUpGateWgrad) { mt = 2 * ((h + R - 1) / R); nt = (d + 255) / 256; nk = cp / 64; }
 }
 
-template <int KIND>
+// Tile `tile` of the sorted list.  128-row tiles: the tile itself.  256-row tiles: its first half (rows
+// m0 .. m0+127); a_boxes_peer carries the second half's boxes.
+template <int KIND, bool WIDE>
 __device__ __forceinline__ Tile decode_tile(const TcParams &prm, const SmemTail *st, int tile, int &cursor)
 {
     const int N = prm.meta.N, d = prm.meta.d;
@@ -309,7 +361,7 @@ __device__ __forceinline__ Tile decode_tile(const TcParams &prm, const SmemTail 
     t.cp = prm.poffsets[t.e + 1] - t.prow0;
     t.pbase = (int)(prm.ebase[t.e] >> 6);
     int mt, nt, nk;
-    expert_shape<KIND>(t.cp, t.h, d, mt, nt, nk);
+    expert_shape<KIND, WIDE>(t.cp, t.h, d, mt, nt, nk);
     const int local = tile - st->tstart[cursor];
     // Order of an expert's tiles (the ~148 tiles in flight should share operands through L2):
     // row-block fastest where the column operand is the big one (weights of the up/gate GEMM, Hm
@@ -317,77 +369,116 @@ __device__ __forceinline__ Tile decode_tile(const TcParams &prm, const SmemTail 
     // fit in flight at once (d / 256 = 8 column blocks), so the row operand is read once.
     constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
     int mb, nb;
-    tile_coords<n_fastest>(local, mt, nt, group_row_tiles(d, 128), mb, nb);
+    tile_coords<n_fastest>(local, mt, nt, group_row_tiles(d, Shape<WIDE>::kTileRows), mb, nb);
     t.nk = nk;
     t.which = 0;
-    t.mrows = 128;
+    int row_extent;                       // extent of the tile's row dimension for this expert
+    if constexpr (KIND == TcDownWgrad) row_extent = d;
+    else if constexpr (KIND == TcUpGateWgrad) { row_extent = t.h; t.which = mb & 1; mb >>= 1; }
+    else row_extent = t.cp;
+    t.m0 = mb * Shape<WIDE>::kTileRows;
+    t.mrows = max(0, min(128, row_extent - t.m0));
+    t.a_boxes = t.mrows / 64;
+    t.a_boxes_peer = WIDE ? max(0, min(128, row_extent - t.m0 - 128)) / 64 : 0;
     if constexpr (KIND == TcUpGate) {
-        t.m0 = mb * 128; t.n0 = nb * 128; t.ncols = min(128, t.h - t.n0);
-        t.n_mma = 2 * t.ncols; t.a_boxes = 2; t.b_boxes = t.n_mma / 64;
-    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
-        t.m0 = mb * 128; t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
-        t.n_mma = t.ncols; t.a_boxes = 2; t.b_boxes = t.ncols / 64;
-    } else if constexpr (KIND == TcDownDgrad || KIND == TcDownWgrad) {
-        t.m0 = mb * 128; t.n0 = nb * 256; t.ncols = min(256, t.h - t.n0);
-        t.n_mma = t.ncols; t.a_boxes = 2; t.b_boxes = t.ncols / 64;
+        t.n0 = nb * 128; t.ncols = min(128, t.h - t.n0);
+        t.n_mma = 2 * t.ncols; t.b_boxes = t.n_mma / 64;
+    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad) {
+        t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
+        t.n_mma = t.ncols; t.b_boxes = t.ncols / 64;
     } else {
-        t.which = mb & 1;
-        t.m0 = (mb >> 1) * 128; t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
-        t.mrows = min(128, t.h - t.m0);
-        t.n_mma = t.ncols; t.a_boxes = t.mrows / 64; t.b_boxes = t.ncols / 64;
+        t.n0 = nb * 256; t.ncols = min(256, t.h - t.n0);
+        t.n_mma = t.ncols; t.b_boxes = t.ncols / 64;
     }
     return t;
 }
 
-// TMA loads of k-block kb of a tile into one stage.
+__device__ __forceinline__ Tile second_half(const Tile &t)
+{
+    Tile u = t;
+    u.m0 = t.m0 + 128;
+    u.a_boxes = t.a_boxes_peer;
+    u.mrows = 64 * t.a_boxes_peer;
+    return u;
+}
+
+// Row-operand boxes of one 128-row half of k-block kb.
 template <int KIND>
-__device__ __forceinline__ void issue_loads(const TcMaps &maps, const Tile &t, int kb, uint32_t a_dst, uint32_t b_dst,
-                                            uint32_t bar)
+__device__ __forceinline__ void load_rows(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
 {
     if constexpr (KIND == TcUpGate) {
-        tma_load_rows(a_dst, &maps.xp, &maps.xp128, bar, kb * 64, t.prow0 + t.m0, 2);
-        const int nb = t.ncols / 64;
-        tma_load_rows(b_dst, &maps.wgate, &maps.wgate128, bar, kb * 64, t.ho + t.n0, nb);
-        tma_load_rows(b_dst + nb * kBoxBytes, &maps.wup, &maps.wup128, bar, kb * 64, t.ho + t.n0, nb);
+        tma_load_rows(dst, &maps.xp, &maps.xp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
     } else if constexpr (KIND == TcDown) {
-        tma_load_rows(a_dst, &maps.hm, &maps.hm128, bar, 0, t.pbase + kb * t.cp + t.m0, 2);
-        tma_load_rows(b_dst, &maps.wdown, &maps.wdown128, bar, t.ho + kb * 64, t.n0, t.b_boxes);
+        tma_load_rows(dst, &maps.hm, &maps.hm128, bar, 0, t.pbase + kb * t.cp + t.m0, t.a_boxes);
     } else if constexpr (KIND == TcDownDgrad) {
-        tma_load_rows(a_dst, &maps.dyp, &maps.dyp128, bar, kb * 64, t.prow0 + t.m0, 2);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + 64 * i, kb * 64);
+        tma_load_rows(dst, &maps.dyp, &maps.dyp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
     } else if constexpr (KIND == TcDownWgrad) {
-        for (int i = 0; i < 2; ++i) tma_load_2d(a_dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
+        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
+    } else if constexpr (KIND == TcUpGateDgrad) {
+        const int half = t.h / 64;
+        const bool second = kb >= half;
+        const int kk = second ? kb - half : kb;
+        tma_load_rows(dst, second ? &maps.db : &maps.da, second ? &maps.db128 : &maps.da128, bar, 0,
+                      t.pbase + kk * t.cp + t.m0, t.a_boxes);
+    } else {
+        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d(dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
+    }
+}
+
+// Column-operand boxes of k-block kb of a tile.
+template <int KIND>
+__device__ __forceinline__ void load_cols(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
+{
+    if constexpr (KIND == TcUpGate) {
+        const int nb = t.ncols / 64;
+        tma_load_rows(dst, &maps.wgate, &maps.wgate128, bar, kb * 64, t.ho + t.n0, nb);
+        tma_load_rows(dst + nb * kBoxBytes, &maps.wup, &maps.wup128, bar, kb * 64, t.ho + t.n0, nb);
+    } else if constexpr (KIND == TcDown) {
+        tma_load_rows(dst, &maps.wdown, &maps.wdown128, bar, t.ho + kb * 64, t.n0, t.b_boxes);
+    } else if constexpr (KIND == TcDownDgrad) {
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + 64 * i, kb * 64);
+    } else if constexpr (KIND == TcDownWgrad) {
         for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d(b_dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + (t.n0 / 64 + i) * t.cp + kb * 64);
+            tma_load_2d(dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + (t.n0 / 64 + i) * t.cp + kb * 64);
     } else if constexpr (KIND == TcUpGateDgrad) {
         const int half = t.h / 64;
         const bool second = kb >= half;
         const int kk = second ? kb - half : kb;
         const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
-        tma_load_rows(a_dst, second ? &maps.db : &maps.da, second ? &maps.db128 : &maps.da128, bar, 0,
-                      t.pbase + kk * t.cp + t.m0, 2);
-        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(b_dst + i * kBoxBytes, bm, bar, t.n0 + 64 * i, t.ho + kk * 64);
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, bm, bar, t.n0 + 64 * i, t.ho + kk * 64);
     } else {
-        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d(b_dst + i * kBoxBytes, &maps.xp, bar, t.n0 + 64 * i, t.prow0 + kb * 64);
+        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.xp, bar, t.n0 + 64 * i, t.prow0 + kb * 64);
     }
 }
 
-// A warp's 32 threads each hold 32 bf16 values of their own row (64 bytes); the rows are
-// `row_stride` elements apart in global memory.  Storing (or loading) them row by row would touch
-// 32 lines with 16 bytes each per instruction, so the chunk is transposed through shared memory:
-// afterwards four neighbouring lanes cover the 64 bytes of one row and an instruction moves eight
-// whole 64-byte row segments.  `own` points at this thread's own row chunk.
-// rows_valid: rows of this warp (0..32, counted from the warp's first row) that may be written.
-// Byte offset of 16-byte piece q of row r in a warp's staging buffer.  Rows are 64 bytes; the piece index is
+// ---------------------------------------------------------------------------
+// Epilogue helpers.  A warp's 32 threads each hold 32 values of their own row.
+// ---------------------------------------------------------------------------
+// Byte offset of 16-byte piece q of row r in a warp's 2 KB buffer.  Rows are 64 bytes; the piece index is
 // XORed with (r / 2) % 4, so that both access patterns are free of bank conflicts: eight lanes writing the
 // same piece of eight consecutive rows, and eight lanes reading all pieces of two consecutive rows.
 __device__ __forceinline__ int epi_piece(int r, int q) { return r * kEpiRowBytes + ((q ^ ((r >> 1) & 3)) << 4); }
 
+__device__ __forceinline__ void pack_bf16x32(const float (&v)[32], uint4 (&w4)[4])
+{
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
+            w[i] = *reinterpret_cast<uint32_t *>(&t);
+        }
+        w4[q] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+// Row-by-row stores of a warp's chunk would touch 32 lines with 16 bytes each per instruction, so the chunk is
+// transposed through shared memory: afterwards four neighbouring lanes cover the 64 bytes of one row and an
+// instruction moves eight whole 64-byte row segments.  `own` points at this thread's own row chunk.
+// rows_valid: rows of this warp (0..32, counted from the warp's first row) that may be written.
 __device__ __forceinline__ void store_u4x4_staged(unsigned char *stg, int lane, unsigned char *own, long long row_stride_bytes,
                                                   const uint4 (&w)[4], int rows_valid)
 {
@@ -408,16 +499,7 @@ __device__ __forceinline__ void store_bf16x32_staged(unsigned char *stg, int lan
                                                      const float (&v)[32], int rows_valid = 32)
 {
     uint4 w4[4];
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            __nv_bfloat162 t = __floats2bfloat162_rn(v[q * 8 + 2 * i], v[q * 8 + 2 * i + 1]);
-            w[i] = *reinterpret_cast<uint32_t *>(&t);
-        }
-        w4[q] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
+    pack_bf16x32(v, w4);
     store_u4x4_staged(stg, lane, reinterpret_cast<unsigned char *>(own), row_stride * 2, w4, rows_valid);
 }
 
@@ -433,6 +515,40 @@ __device__ __forceinline__ void store_f32x32_staged(unsigned char *stg, int lane
             w4[q] = make_uint4(__float_as_uint(v[hh * 16 + 4 * q]), __float_as_uint(v[hh * 16 + 4 * q + 1]),
                                __float_as_uint(v[hh * 16 + 4 * q + 2]), __float_as_uint(v[hh * 16 + 4 * q + 3]));
         store_u4x4_staged(stg, lane, reinterpret_cast<unsigned char *>(own + hh * 16), row_stride * 4, w4, rows_valid);
+    }
+}
+
+__device__ __forceinline__ void red_add_f32x4(float *addr, const uint4 &v)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                 ::"l"(addr), "f"(__uint_as_float(v.x)), "f"(__uint_as_float(v.y)), "f"(__uint_as_float(v.z)),
+                   "f"(__uint_as_float(v.w))
+                 : "memory");
+}
+
+// The warp's 32 rows x 32 fp32 values are added into rows tok (one per lane; -1: no row) of a [T, row_stride]
+// fp32 matrix at column col0: the same transposition, then 16-byte reductions.  With at most two rows added
+// into a zeroed element the result does not depend on their order (0 + a + b == 0 + b + a).
+__device__ __forceinline__ void red_f32x32_staged(unsigned char *stg, int lane, float *base, long long row_stride, int tok,
+                                                  int col0, const float (&v)[32])
+{
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4 *>(stg + epi_piece(lane, q)) =
+                make_uint4(__float_as_uint(v[hh * 16 + 4 * q]), __float_as_uint(v[hh * 16 + 4 * q + 1]),
+                           __float_as_uint(v[hh * 16 + 4 * q + 2]), __float_as_uint(v[hh * 16 + 4 * q + 3]));
+        __syncwarp();
+        const int q = lane & 3;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int rr = 8 * j + (lane >> 2);
+            const int tk = __shfl_sync(0xFFFFFFFFu, tok, rr);
+            const uint4 val = *reinterpret_cast<const uint4 *>(stg + epi_piece(rr, q));
+            if (tk >= 0) red_add_f32x4(base + (long long)tk * row_stride + col0 + hh * 16 + q * 4, val);
+        }
+        __syncwarp();
     }
 }
 
@@ -464,35 +580,55 @@ __device__ __forceinline__ void untranspose_rows(unsigned char *stg, int lane, c
 }
 
 // Called before the accumulator of a tile is ready: asks L2 for what the epilogue will read from
-// global memory (only the down dgrad reads: the two saved SwiGLU factors of its row).
-template <int KIND>
-__device__ __forceinline__ void epilogue_prefetch(const TcParams &prm, const Tile &t, int row, int c_begin, int c_end)
+// global memory (only the down dgrad reads: the saved SwiGLU factors of its row, and Hm for the row dot).
+// The tile's 32-column chunks are split into NQ contiguous runs, one per warp of the lane quadrant.
+template <int NQ>
+__device__ __forceinline__ void chunk_range(int ncols, int cq, int &c_begin, int &c_end)
+{
+    const int per = ((ncols >> 5) + NQ - 1) / NQ;
+    c_begin = min(ncols, cq * per * 32);
+    c_end = min(ncols, c_begin + per * 32);
+}
+
+template <int KIND, int VAR, int NQ>
+__device__ __forceinline__ void epilogue_prefetch(const TcParams &prm, const Tile &t, int row, int cq)
 {
     if constexpr (KIND == TcDownDgrad) {
-        for (int c = c_begin; c < c_end; c += 64) {      // one 128-byte line per array covers two 32-column chunks
+        int c_begin, c_end;
+        chunk_range<NQ>(t.ncols, cq, c_begin, c_end);
+        for (int c = c_begin; c < c_end; c += 32) {
             const int col = t.n0 + c;
-            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6);
+            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
             asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.sp + idx));
             asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.sq + idx));
+            if constexpr (VAR == 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.hm + idx));
         }
     }
 }
 
-// Epilogue of one tile for one thread: accumulator row `row`, columns [c_begin, c_end).
-template <int KIND>
-__device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t, uint32_t tacc, int row, int c_begin,
-                                             int c_end, unsigned char *stg)
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// Epilogue of one 128-row (half) tile for one thread: accumulator row `row`, run cq of the tile's 32-column
+// chunks (NQ = epilogue warps per TMEM lane quadrant).
+//   VAR = 1 selects the product's fused variant: DownDgrad also writes the partial row dot of its
+//   accumulator with Hm (for dg); Down and UpGateDgrad add their rows into fp32 [T, d] token rows.
+template <int KIND, int VAR, int NQ>
+__device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t, uint32_t tacc, int row, int lane, int cq,
+                                             unsigned char *stg)
 {
-    const int lane = row & 31;
     const int d = prm.meta.d, S = prm.meta.S;
     const bool have_acc = t.nk > 0;
+    int c_first, c_end;
+    chunk_range<NQ>(t.ncols, cq, c_first, c_end);
+    constexpr int c_step = 32;
     auto panel_index = [&](int c) {
         const int col = t.n0 + c;
         return ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
     };
     if constexpr (KIND == TcUpGate) {
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
-        for (int c = c_begin; c < c_end; c += 32) {
+        for (int c = c_first; c < c_end; c += c_step) {
             uint32_t ra[32], rb[32];
             tmem_ld32(tacc + c, ra);
             tmem_ld32(tacc + t.ncols + c, rb);
@@ -521,40 +657,74 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             store_bf16x32_staged(stg, lane, prm.hm + idx, 64, hm);
         }
     } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
-        float *out = (KIND == TcDown ? prm.o : prm.dxp) + (size_t)(t.prow0 + t.m0 + row) * d + t.n0;
-        for (int c = c_begin; c < c_end; c += 32) {
-            uint32_t r[32];
-            float v[32];
-            tmem_ld32(tacc + c, r);
-            tmem_ld_wait();
+        if constexpr (VAR == 1) {
+            int tok = prm.ptoken_of[t.prow0 + t.m0 + row];
+            if (tok >= prm.T) {                      // not a token of this batch: recorded, row skipped
+                atomicMax(prm.status, kDevBounds);
+                tok = -1;
+            }
+            for (int c = c_first; c < c_end; c += c_step) {
+                uint32_t r[32];
+                float v[32];
+                tmem_ld32(tacc + c, r);
+                tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-            store_f32x32_staged(stg, lane, out + c, d, v);
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                red_f32x32_staged(stg, lane, prm.scatter_out, d, tok, t.n0 + c, v);
+            }
+        } else {
+            float *out = (KIND == TcDown ? prm.o : prm.dxp) + (size_t)(t.prow0 + t.m0 + row) * d + t.n0;
+            for (int c = c_first; c < c_end; c += c_step) {
+                uint32_t r[32];
+                float v[32];
+                tmem_ld32(tacc + c, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                store_f32x32_staged(stg, lane, out + c, d, v);
+            }
         }
     } else if constexpr (KIND == TcDownDgrad) {
         // dA = dHm * sp, dB = dHm * sq with dHm = gate * acc; the saved factors of the next
         // chunk are fetched while this one is computed
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
-        uint4 praw[4], qraw[4];            // transposed: entry j belongs to row 8j + lane/4 of this warp
-        {
-            const size_t idx = panel_index(c_begin);
+        float rowdot = 0.f;                // VAR 1: sum over this thread's columns of acc * Hm
+        uint4 praw[4], qraw[4], hraw[4];   // transposed: entry j belongs to row 8j + lane/4 of this warp
+        if (c_first < c_end) {
+            const size_t idx = panel_index(c_first);
             load_bf16x32_transposed(prm.sp + idx, 64, lane, praw);
             load_bf16x32_transposed(prm.sq + idx, 64, lane, qraw);
+            if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + idx, 64, lane, hraw);
         }
-        for (int c = c_begin; c < c_end; c += 32) {
+        for (int c = c_first; c < c_end; c += c_step) {
             uint32_t r[32];
             tmem_ld32(tacc + c, r);
-            uint4 pn[4], qn[4];
-            const bool more = c + 32 < c_end;
+            uint4 pn[4], qn[4], hn[4];
+            const bool more = c + c_step < c_end;
             if (more) {
-                const size_t nidx = panel_index(c + 32);
+                const size_t nidx = panel_index(c + c_step);
                 load_bf16x32_transposed(prm.sp + nidx, 64, lane, pn);
                 load_bf16x32_transposed(prm.sq + nidx, 64, lane, qn);
+                if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + nidx, 64, lane, hn);
             }
             uint4 pown[4], qown[4];
             untranspose_rows(stg, lane, praw, pown);
             untranspose_rows(stg, lane, qraw, qown);
             tmem_ld_wait();
+            if constexpr (VAR == 1) {
+                uint4 hown[4];
+                untranspose_rows(stg, lane, hraw, hown);
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const uint32_t hw[4] = {hown[q4].x, hown[q4].y, hown[q4].z, hown[q4].w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int e0 = q4 * 8 + 2 * i;
+                        rowdot = fmaf(__uint_as_float(r[e0]), bf16_lo(hw[i]), rowdot);
+                        rowdot = fmaf(__uint_as_float(r[e0 + 1]), bf16_hi(hw[i]), rowdot);
+                    }
+                }
+            }
             const size_t idx = panel_index(c);
             float da[32], db[32];
 #pragma unroll
@@ -565,10 +735,10 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
                 for (int i = 0; i < 4; ++i) {
                     const int e0 = q4 * 8 + 2 * i;
                     const float dh0 = gate * __uint_as_float(r[e0]), dh1 = gate * __uint_as_float(r[e0 + 1]);
-                    da[e0] = dh0 * __uint_as_float(pw[i] << 16);
-                    da[e0 + 1] = dh1 * __uint_as_float(pw[i] & 0xFFFF0000u);
-                    db[e0] = dh0 * __uint_as_float(qw[i] << 16);
-                    db[e0 + 1] = dh1 * __uint_as_float(qw[i] & 0xFFFF0000u);
+                    da[e0] = dh0 * bf16_lo(pw[i]);
+                    da[e0 + 1] = dh1 * bf16_hi(pw[i]);
+                    db[e0] = dh0 * bf16_lo(qw[i]);
+                    db[e0 + 1] = dh1 * bf16_hi(qw[i]);
                 }
             }
             store_bf16x32_staged(stg, lane, prm.da + idx, 64, da);
@@ -576,11 +746,18 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             if (more) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) { praw[i] = pn[i]; qraw[i] = qn[i]; }
+                if constexpr (VAR == 1) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) hraw[i] = hn[i];
+                }
             }
         }
+        // one partial per (row, 256-column tile, half of the columns); a warp without a chunk writes its zero
+        if constexpr (VAR == 1)
+            prm.dg_part[(size_t)((t.n0 >> 8) * 2 + cq) * prm.Pmax + t.prow0 + t.m0 + row] = rowdot;
     } else if constexpr (KIND == TcDownWgrad) {
         const size_t oidx = (size_t)(t.m0 + row) * S + t.ho + t.n0;
-        for (int c = c_begin; c < c_end; c += 32) {
+        for (int c = c_first; c < c_end; c += c_step) {
             float v[32];
             if (have_acc) {
                 uint32_t r[32];
@@ -592,13 +769,14 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
 #pragma unroll
                 for (int i = 0; i < 32; ++i) v[i] = 0.f;
             }
-            if (prm.out_f32) store_f32x32_staged(stg, lane, reinterpret_cast<float *>(prm.dw_down) + oidx + c, S, v);
-            else store_bf16x32_staged(stg, lane, prm.dw_down + oidx + c, S, v);
+            const int rows_valid = t.mrows - (row - lane);
+            if (prm.out_f32) store_f32x32_staged(stg, lane, reinterpret_cast<float *>(prm.dw_down) + oidx + c, S, v, rows_valid);
+            else store_bf16x32_staged(stg, lane, prm.dw_down + oidx + c, S, v, rows_valid);
         }
     } else {
         __nv_bfloat16 *obase = t.which ? prm.dw_up : prm.dw_gate;
         const size_t oidx = (size_t)(t.ho + t.m0 + row) * d + t.n0;
-        for (int c = c_begin; c < c_end; c += 32) {
+        for (int c = c_first; c < c_end; c += c_step) {
             float v[32];
             if (have_acc) {
                 uint32_t r[32];
@@ -617,92 +795,197 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
     }
 }
 
+// ---------------------------------------------------------------------------
+// Schedule: experts by decreasing K, tiles of an expert contiguous.  `key` and
+// `ntile` are scratch arrays of kMaxExperts ints (the epilogue buffers serve).
+// ---------------------------------------------------------------------------
+template <int KIND, bool WIDE>
+__device__ __forceinline__ void build_schedule(const TcParams &prm, SmemTail *st, int *key, int *ntile, int tid)
+{
+    const int N = prm.meta.N, d = prm.meta.d;
+    for (int e = tid; e < N; e += kThreads) {
+        const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
+        const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
+        int mt, nt, nk;
+        expert_shape<KIND, WIDE>(cp, h, d, mt, nt, nk);
+        // a group outside the padded row space (or not padded to whole tiles) is recorded and gets no tiles
+        const bool sane = prm.poffsets[e] >= 0 && cp >= 0 && prm.poffsets[e + 1] <= prm.Pmax && (prm.poffsets[e] & 127) == 0 &&
+                          (cp & 127) == 0;
+        if (!sane && blockIdx.x == 0) atomicMax(prm.status, kDevBounds);
+        ntile[e] = sane ? mt * nt : 0;
+        key[e] = nk;
+    }
+    __syncthreads();
+    for (int e = tid; e < N; e += kThreads) {
+        int rank = 0;
+        const int ke = key[e];
+        for (int f = 0; f < N; ++f) {
+            const int kf = key[f];
+            rank += (kf > ke) || (kf == ke && f < e);
+        }
+        st->order[rank] = (unsigned short)e;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int acc = 0;
+        for (int i = 0; i < N; ++i) { st->tstart[i] = acc; acc += ntile[st->order[i]]; }
+        st->tstart[N] = acc;
+    }
+}
+
+// The tile warp's loop: takes tile after tile from the global counter and hands each to the three working roles
+// through the queue; ends with -1 when the list is exhausted.  It stays one tile ahead of the TMA leader, the
+// most advanced role (tq_taken): enough to hide the counter's round trip, and no more, because a tile taken
+// early is a tile another CTA cannot take.
+__device__ __forceinline__ void hand_out_tiles(const TcParams &prm, SmemTail *st, int total, const WaitCtx &w)
+{
+    for (int it = 0;; ++it) {
+        const int slot = it & (kTileQ - 1);
+        const uint32_t ph = (uint32_t)(it / kTileQ) & 1u;
+        if (it > 0 && !mbar_wait(smem_u32(&st->tq_taken), (uint32_t)(it - 1) & 1u, w)) return;   // the leader has started on tile it - 1
+        if (!mbar_wait(smem_u32(&st->tq_empty[slot]), ph ^ 1u, w)) return;
+        int tile = atomicAdd(prm.tile_counter, 1);
+        if (tile >= total) tile = -1;
+        st->tile_q[slot] = tile;
+        mbar_arrive(smem_u32(&st->tq_full[slot]));
+        if (tile < 0) return;
+    }
+}
+
+// Consumer side: the it-th tile of this CTA (-1: no more), not yet released.
 template <int KIND>
+__device__ __forceinline__ int peek_tile(const TcParams &prm, SmemTail *st, int it, int total, const WaitCtx &w, bool &ok)
+{
+    if (!prm.dynamic) {
+        const int tile = dealt_tile<KIND>(it, blockIdx.x, gridDim.x);
+        return tile >= total ? -1 : tile;
+    }
+    const int slot = it & (kTileQ - 1);
+    const uint32_t ph = (uint32_t)(it / kTileQ) & 1u;
+    if (!mbar_wait(smem_u32(&st->tq_full[slot]), ph, w)) { ok = false; return -1; }
+    return *reinterpret_cast<volatile int *>(&st->tile_q[slot]);
+}
+__device__ __forceinline__ void release_tile(const TcParams &prm, SmemTail *st, int it)
+{
+    if (prm.dynamic) mbar_arrive(smem_u32(&st->tq_empty[it & (kTileQ - 1)]));
+}
+
+// ---------------------------------------------------------------------------
+// The kernel.  WIDE: 256-row tiles (two halves sharing the column operand; both
+// accumulators belong to the tile).  VAR 1: the product's fused variant -
+// UpGate gathers its rows from x by token index (every lane of the producer
+// warp issues one four-row gather per half and k-block), DownDgrad writes row
+// dots for dg, Down / UpGateDgrad add into token rows.
+// ---------------------------------------------------------------------------
+template <int KIND, bool WIDE, int VAR>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
 {
+    constexpr int NQ = kEpiWarps / 4;            // epilogue warps per TMEM lane quadrant
+    using Sh = Shape<WIDE>;
+    constexpr int kStages = Sh::kStages;
+    constexpr int kStageBytes = Sh::kStageBytes;
+    constexpr bool kGather = (KIND == TcUpGate && VAR == 1);
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
     unsigned char *smem = smem_raw + pad;
     const uint32_t stage_base = raw + pad;
-    SmemTail *st = reinterpret_cast<SmemTail *>(smem + (size_t)kStages * kStageBytes);
+    unsigned char *epi_bufs = smem + (size_t)kStages * kStageBytes;
+    SmemTail *st = reinterpret_cast<SmemTail *>(epi_bufs + kEpiBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int N = prm.meta.N, d = prm.meta.d;
 
-    // ---- schedule: experts by decreasing K, tiles of an expert contiguous ----
-    for (int e = tid; e < N; e += kThreads) {
-        const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
-        const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
-        int mt, nt, nk;
-        expert_shape<KIND>(cp, h, d, mt, nt, nk);
-        st->ntile[e] = mt * nt;
-        st->key[e] = nk;
-    }
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(smem_u32(&st->full[s]), 1);
             mbar_init(smem_u32(&st->empty[s]), 1);
         }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&st->tmem_full[a]), 1);
-            mbar_init(smem_u32(&st->tmem_empty[a]), 256);
+        mbar_init(smem_u32(&st->tmem_full[0]), 1);
+        mbar_init(smem_u32(&st->tmem_full[1]), 1);
+        mbar_init(smem_u32(&st->tmem_empty[0]), 32 * kEpiWarps);
+        mbar_init(smem_u32(&st->tmem_empty[1]), 32 * kEpiWarps);
+        mbar_init(smem_u32(&st->tq_taken), 1);
+        for (int s = 0; s < kTileQ; ++s) {
+            mbar_init(smem_u32(&st->tq_full[s]), 1);
+            mbar_init(smem_u32(&st->tq_empty[s]), 2 + kEpiWarps);   // the TMA leader, the MMA thread and one lane of each epilogue warp
         }
         st->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    __syncthreads();
-    for (int e = tid; e < N; e += kThreads) {
-        int rank = 0;
-        const int ke = st->key[e];
-        for (int f = 0; f < N; ++f) {
-            const int kf = st->key[f];
-            rank += (kf > ke) || (kf == ke && f < e);
-        }
-        st->order[rank] = e;
-    }
+    build_schedule<KIND, WIDE>(prm, st, reinterpret_cast<int *>(epi_bufs), reinterpret_cast<int *>(epi_bufs) + kMaxExperts, tid);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&st->tmem_base)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    __syncthreads();
-    if (tid == 0) {
-        int acc = 0;
-        for (int i = 0; i < N; ++i) { st->tstart[i] = acc; acc += st->ntile[st->order[i]]; }
-        st->tstart[N] = acc;
-    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = st->tmem_base;
-    const int total_tiles = st->tstart[N];
-    volatile int *abort_flag = &st->abort_flag;
+    const int total_tiles = st->tstart[prm.meta.N];
+    const WaitCtx wc{&st->abort_flag, prm.status, prm.wait_limit_ns};
 
     if (warp == 0) {
         // ===================== TMA producer =====================
-        if (lane == 0) {
+        if (kGather || lane == 0) {
             int stage = 0, cursor = 0;
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
-            for (int rnd = 0, tile = dealt_tile<KIND>(0, blockIdx.x, gridDim.x); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, blockIdx.x, gridDim.x)) {
-                const Tile t = decode_tile<KIND>(prm, st, tile, cursor);
-                const uint32_t bytes = (uint32_t)(t.a_boxes + t.b_boxes) * kBoxBytes;
-                for (int kb = 0; kb < t.nk; ++kb) {
-                    if (!mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
+            for (int it = 0; ok; ++it) {
+                int tile = -1;
+                if (lane == 0) {
+                    tile = peek_tile<KIND>(prm, st, it, total_tiles, wc, ok);
+                    if (ok) {
+                        release_tile(prm, st, it);
+                        if (prm.dynamic) mbar_arrive(smem_u32(&st->tq_taken));
+                    }
+                }
+                if constexpr (kGather) {
+                    tile = __shfl_sync(0xFFFFFFFFu, tile, 0);
+                    ok = __shfl_sync(0xFFFFFFFFu, (int)ok, 0) != 0;
+                }
+                if (!ok || tile < 0 || tile == prm.skip_tile) break;
+                const Tile t0 = decode_tile<KIND, WIDE>(prm, st, tile, cursor);
+                const Tile t1 = second_half(t0);
+                const uint32_t bytes = (uint32_t)(t0.a_boxes + (WIDE ? t1.a_boxes : 0) + t0.b_boxes) * kBoxBytes;
+                int4 tok0 = make_int4(-1, -1, -1, -1), tok1 = make_int4(-1, -1, -1, -1);
+                if constexpr (kGather) {
+                    // rows 4 lane .. 4 lane + 3 of each half: their tokens (pad rows and rows past the group: -1)
+                    const int r0 = t0.prow0 + t0.m0 + 4 * lane;
+                    if (4 * lane < t0.mrows) tok0 = *reinterpret_cast<const int4 *>(prm.ptoken_of + r0);
+                    if (WIDE && 4 * lane < t1.mrows) tok1 = *reinterpret_cast<const int4 *>(prm.ptoken_of + r0 + 128);
+                }
+                for (int kb = 0; kb < t0.nk; ++kb) {
+                    // the leader waits for the stage; with all lanes at work they take its verdict, so that none
+                    // leaves the loop alone
+                    bool got = (lane == 0) ? mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, wc) : true;
+                    if constexpr (kGather) got = __shfl_sync(0xFFFFFFFFu, (int)got, 0) != 0;
+                    if (!got) { ok = false; break; }
                     const uint32_t bar = smem_u32(&st->full[stage]);
-                    mbar_arrive_expect_tx(bar, bytes);
                     const uint32_t a_dst = stage_base + stage * kStageBytes;
-                    issue_loads<KIND>(maps, t, kb, a_dst, a_dst + kARegion, bar);
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(bar, bytes);
+                        if constexpr (!kGather) {
+                            load_rows<KIND>(maps, t0, kb, a_dst, bar);
+                            if constexpr (WIDE) load_rows<KIND>(maps, t1, kb, a_dst + kARegion, bar);
+                        }
+                        load_cols<KIND>(maps, t0, kb, a_dst + Sh::kRowRegion, bar);
+                    }
+                    if constexpr (kGather) {
+                        __syncwarp();                         // the byte count is posted before any copy can complete
+                        if (4 * lane < 64 * t0.a_boxes)
+                            tma_gather4(a_dst + lane * 512, &maps.xg, bar, kb * 64, tok0.x, tok0.y, tok0.z, tok0.w);
+                        if (WIDE && 4 * lane < 64 * t1.a_boxes)
+                            tma_gather4(a_dst + kARegion + lane * 512, &maps.xg, bar, kb * 64, tok1.x, tok1.y, tok1.z, tok1.w);
+                    }
                     ++issued;
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!ok) {
+            if (!ok && lane == 0) {
                 // let the copies already issued land before the CTA leaves: wait (bounded) for
                 // the current phase of every stage that has had a load
                 const int n = issued < kStages ? (int)issued : kStages;
@@ -710,67 +993,131 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
                     int s = stage - i;
                     uint32_t ph = phase;
                     if (s < 0) { s += kStages; ph ^= 1u; }
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(smem_u32(&st->full[s]), ph) && global_ns() - t0 < kWaitLimitNs) {}
+                    const unsigned long long tb = global_ns();
+                    while (!mbar_try_wait(smem_u32(&st->full[s]), ph) && global_ns() - tb < prm.wait_limit_ns) {}
                 }
             }
         }
     } else if (warp == 1) {
         // ===================== MMA issuer =====================
         if (lane == 0) {
-            int stage = 0, cursor = 0, it = 0;
+            int stage = 0, cursor = 0;
             uint32_t phase = 0;
+            uint32_t use0 = 0, use1 = 0;         // WIDE: how often each accumulator has been handed to the epilogue
             bool ok = true;
             constexpr bool a_mn = KindTraits<KIND>::a_mn, b_mn = KindTraits<KIND>::b_mn;
             constexpr uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
             constexpr uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
-            for (int rnd = 0, tile = dealt_tile<KIND>(0, blockIdx.x, gridDim.x); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, blockIdx.x, gridDim.x), ++it) {
-                const Tile t = decode_tile<KIND>(prm, st, tile, cursor);
-                const int acc = it & 1;
-                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t tacc = tmem_base + (uint32_t)(acc * kAccCols);
-                const uint32_t idesc = make_idesc(a_mn, b_mn, t.n_mma);
-                for (int kb = 0; kb < t.nk; ++kb) {
-                    if (!mbar_wait(smem_u32(&st->full[stage]), phase, abort_flag, prm.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = stage_base + stage * kStageBytes;
-                    const uint64_t adesc = make_desc(a_addr, a_mn);
-                    const uint64_t bdesc = make_desc(a_addr + kARegion, b_mn);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_bf16(tacc, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
-                                  (kb > 0 || ks > 0) ? 1u : 0u);
-                    umma_commit(smem_u32(&st->empty[stage]));   // frees the stage once these MMAs have read it
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                }
+            for (int it = 0; ok; ++it) {
+                const int tile = peek_tile<KIND>(prm, st, it, total_tiles, wc, ok);
                 if (!ok) break;
-                if (t.nk > 0) umma_commit(smem_u32(&st->tmem_full[acc]));
-                else mbar_arrive(smem_u32(&st->tmem_full[acc]));
+                release_tile(prm, st, it);
+                if (tile < 0) break;
+                const Tile t = decode_tile<KIND, WIDE>(prm, st, tile, cursor);
+                const uint32_t idesc = make_idesc(a_mn, b_mn, t.n_mma);
+                if constexpr (!WIDE) {
+                    const int acc = it & 1;
+                    const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                    if (!mbar_wait(smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, wc)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t tacc = tmem_base + (uint32_t)(acc * kAccCols);
+                    for (int kb = 0; kb < t.nk; ++kb) {
+                        if (!mbar_wait(smem_u32(&st->full[stage]), phase, wc)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = stage_base + stage * kStageBytes;
+                        const uint64_t adesc = make_desc(a_addr, a_mn);
+                        const uint64_t bdesc = make_desc(a_addr + kARegion, b_mn);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_bf16(tacc, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
+                                      (kb > 0 || ks > 0) ? 1u : 0u);
+                        umma_commit(smem_u32(&st->empty[stage]));   // frees the stage once these MMAs have read it
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    if (t.nk > 0) umma_commit(smem_u32(&st->tmem_full[acc]));
+                    else mbar_arrive(smem_u32(&st->tmem_full[acc]));
+                } else {
+                    const bool two = t.a_boxes_peer > 0;
+                    if (!mbar_wait(smem_u32(&st->tmem_empty[0]), (use0 & 1u) ^ 1u, wc)) { ok = false; break; }
+                    tc_fence_after();
+                    for (int kb = 0; kb < t.nk; ++kb) {
+                        if (!mbar_wait(smem_u32(&st->full[stage]), phase, wc)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t a_addr = stage_base + stage * kStageBytes;
+                        const uint64_t adesc0 = make_desc(a_addr, a_mn);
+                        const uint64_t adesc1 = make_desc(a_addr + kARegion, a_mn);
+                        const uint64_t bdesc = make_desc(a_addr + Sh::kRowRegion, b_mn);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_bf16(tmem_base, adesc0 + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
+                                      (kb > 0 || ks > 0) ? 1u : 0u);
+                        if (two) {
+                            if (kb == 0) {
+                                // the second accumulator may still be draining: the first half's MMAs above are already queued
+                                if (!mbar_wait(smem_u32(&st->tmem_empty[1]), (use1 & 1u) ^ 1u, wc)) { ok = false; break; }
+                                tc_fence_after();
+                            }
+#pragma unroll
+                            for (int ks = 0; ks < 4; ++ks)
+                                umma_bf16(tmem_base + kAccCols, adesc1 + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step),
+                                          idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                        }
+                        umma_commit(smem_u32(&st->empty[stage]));
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    if (t.nk > 0) umma_commit(smem_u32(&st->tmem_full[0]));
+                    else mbar_arrive(smem_u32(&st->tmem_full[0]));
+                    ++use0;
+                    if (two) ++use1;
+                }
             }
         }
+    } else if (warp == 2) {
+        // ===================== tile hand-out =====================
+        if (lane == 0 && prm.dynamic) hand_out_tiles(prm, st, total_tiles, wc);
     } else {
-        // ===================== epilogue (warps 2..9) =====================
+        // ===================== epilogue (warps 3 .. 10) =====================
         const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
-        const int half = (warp - 2) >> 2;          // which half of the tile's columns
+        const int cq = (warp - kFirstEpiWarp) >> 2;   // which of the quadrant's two warps: the first or second half of the columns
         const int row = quad * 32 + lane;
-        int cursor = 0, it = 0;
+        unsigned char *stg = epi_bufs + (warp - kFirstEpiWarp) * kEpiBufBytes;
+        int cursor = 0;
         bool ok = true;
-        for (int rnd = 0, tile = dealt_tile<KIND>(0, blockIdx.x, gridDim.x); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, blockIdx.x, gridDim.x), ++it) {
-            const Tile t = decode_tile<KIND>(prm, st, tile, cursor);
-            const int acc = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            const int chalf = t.ncols >> 1;            // a multiple of 32: ncols is a multiple of 64
-            epilogue_prefetch<KIND>(prm, t, row, half * chalf, (half + 1) * chalf);
-            if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, prm.status)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
-            epilogue_row<KIND>(prm, t, tacc, row, half * chalf, (half + 1) * chalf, st->epi_stage[warp - 2]);
-            tc_fence_before();
-            mbar_arrive(smem_u32(&st->tmem_empty[acc]));
+        for (int it = 0; ok; ++it) {
+            const int tile = peek_tile<KIND>(prm, st, it, total_tiles, wc, ok);
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) release_tile(prm, st, it);
+            if (tile < 0) break;
+            const Tile t = decode_tile<KIND, WIDE>(prm, st, tile, cursor);
+            if constexpr (!WIDE) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                epilogue_prefetch<KIND, VAR, NQ>(prm, t, row, cq);
+                if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, wc)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
+                epilogue_row<KIND, VAR, NQ>(prm, t, tacc, row, lane, cq, stg);
+                tc_fence_before();
+                mbar_arrive(smem_u32(&st->tmem_empty[acc]));
+            } else {
+                epilogue_prefetch<KIND, VAR, NQ>(prm, t, row, cq);
+                if (!mbar_wait(smem_u32(&st->tmem_full[0]), (uint32_t)it & 1u, wc)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16);
+                epilogue_row<KIND, VAR, NQ>(prm, t, tacc, row, lane, cq, stg);
+                tc_fence_before();
+                mbar_arrive(smem_u32(&st->tmem_empty[0]));
+                if (t.a_boxes_peer > 0) {
+                    const Tile t1 = second_half(t);
+                    epilogue_prefetch<KIND, VAR, NQ>(prm, t1, row, cq);
+                    epilogue_row<KIND, VAR, NQ>(prm, t1, tacc + kAccCols, row, lane, cq, stg);
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&st->tmem_empty[1]));
+                }
+            }
         }
     }
 
@@ -784,684 +1131,21 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
     }
 }
 
-// ===========================================================================
-// Two-CTA variant (cta_group::2).  A cluster of two CTAs on neighbouring SMs
-// computes one 256-row tile: each CTA stages its own 128 rows of the row
-// operand and HALF of the column operand (so a CTA moves 32 KB per k-block
-// instead of 48 KB), the leader CTA (cluster rank 0) issues tcgen05.mma with
-// M = 256 reading both CTAs' shared memory, and each CTA's TMEM receives the
-// accumulator rows of its own half.  Barrier protocol:
-//   full[s]       leader only; its producer posts the byte count of both CTAs,
-//                 both producers' TMA loads complete on it
-//   empty[s]      one per CTA; tcgen05.commit multicasts to both
-//   tmem_full[a]  one per CTA; tcgen05.commit multicasts to both
-//   tmem_empty[a] leader only; one arrival per epilogue warp of both CTAs
-// ===========================================================================
-constexpr int kStages2 = 6;
-constexpr int kARegion2 = 2 * kBoxBytes;
-constexpr int kBRegion2 = 2 * kBoxBytes;
-constexpr int kStageBytes2 = kARegion2 + kBRegion2;   // 32 KB
-struct SmemTail2 {
-    unsigned char epi_stage[8][kEpiWarpBytes];   // one transposing buffer per epilogue warp
-    unsigned long long full[kStages2], empty[kStages2], tmem_full[2], tmem_empty[2];
-    unsigned int tmem_base;
-    int abort_flag;
-    int order[kMaxExperts];
-    int key[kMaxExperts];
-    int ntile[kMaxExperts];
-    int tstart[kMaxExperts + 1];
-};
-constexpr size_t kSmemBytes2 = 1024 + (size_t)kStages2 * kStageBytes2 + sizeof(SmemTail2);
-
-__device__ __forceinline__ uint32_t cluster_ctarank()
+// Sums the partial row dots of the down dgrad in slot order and divides by the gate:
+// dg[t, j] = <dY_t W_down, Hm_row> / g = <dY_t, E_(t,j)>.  One thread per assignment.
+__global__ void __launch_bounds__(256)
+dg_finish_kernel(LayerMeta m, int Ttok, int Pmax, const int *__restrict__ topk_idx, const float *__restrict__ topk_gate,
+                 const int *__restrict__ prow_of, const float *__restrict__ dg_part, float *__restrict__ dg, int *status)
 {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t leader_bar, int x, int y)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(leader_bar), "r"(x), "r"(y)
-        : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((unsigned short)3) : "memory");
-}
-__device__ __forceinline__ uint32_t make_idesc_pair(bool a_mn, bool b_mn, int n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-}
-
-template <int KIND>
-__device__ __forceinline__ void expert_shape2(int cp, int h, int d, int &mt, int &nt, int &nk)
-{
-    if constexpr (KIND == TcUpGate)      { mt = (cp + 255) / 256; nt = (h + 127) / 128; nk = d / 64; }
-    if constexpr (KIND == TcDown)        { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = h / 64; }
-    if constexpr (KIND == TcDownDgrad)   { mt = (cp + 255) / 256; nt = (h + 255) / 256; nk = d / 64; }
-    if constexpr (KIND == TcDownWgrad)   { mt = (d + 255) / 256;  nt = (h + 255) / 256; nk = cp / 64; }
-    if constexpr (KIND == TcUpGateDgrad) { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = 2 * (h / 64); }
-    if constexpr (KIND == TcUpGateWgrad) { mt = 2 * ((h + 255) / 256); nt = (d + 255) / 256; nk = cp / 64; }
-}
-
-// Tile of this CTA (cluster rank `rank`) inside pair tile `tile`.  Fields as in the one-CTA
-// decode; m0 / mrows / a_boxes describe this CTA's 128-row half, a_boxes_peer the other half,
-// b_boxes and b_off this CTA's half of the column operand, ncols the columns that are stored.
-template <int KIND>
-__device__ __forceinline__ Tile decode_tile2(const TcParams &prm, const SmemTail2 *st, int tile, int &cursor, int rank)
-{
-    const int N = prm.meta.N, d = prm.meta.d;
-    while (cursor + 1 < N && tile >= st->tstart[cursor + 1]) ++cursor;
-    Tile t;
-    t.e = st->order[cursor];
-    t.ho = prm.meta.hoff[t.e];
-    t.h = prm.meta.hoff[t.e + 1] - t.ho;
-    t.prow0 = prm.poffsets[t.e];
-    t.cp = prm.poffsets[t.e + 1] - t.prow0;
-    t.pbase = (int)(prm.ebase[t.e] >> 6);
-    int mt, nt, nk;
-    expert_shape2<KIND>(t.cp, t.h, d, mt, nt, nk);
-    const int local = tile - st->tstart[cursor];
-    constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
-    int mb, nb;
-    tile_coords<n_fastest>(local, mt, nt, group_row_tiles(d, 256), mb, nb);
-    t.nk = nk;
-    t.which = 0;
-    int row_extent;                       // extent of the tile's row dimension for this expert
-    if constexpr (KIND == TcDownWgrad) row_extent = d;
-    else if constexpr (KIND == TcUpGateWgrad) { row_extent = t.h; t.which = mb & 1; mb >>= 1; }
-    else row_extent = t.cp;
-    const int m_pair = mb * 256;
-    t.m0 = m_pair + 128 * rank;
-    t.mrows = max(0, min(128, row_extent - t.m0));
-    const int peer_rows = max(0, min(128, row_extent - (m_pair + 128 * (1 - rank))));
-    t.a_boxes = t.mrows / 64;
-    t.a_boxes_peer = peer_rows / 64;
-    if constexpr (KIND == TcUpGate) {
-        t.n0 = nb * 128; t.ncols = min(128, t.h - t.n0);
-        t.n_mma = 2 * t.ncols; t.b_boxes = t.ncols / 64; t.b_off = 0;
-    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad) {
-        t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
-        t.n_mma = t.ncols; t.b_boxes = t.ncols / 128; t.b_off = rank * (t.ncols / 2);
-    } else {
-        t.n0 = nb * 256; t.ncols = min(256, t.h - t.n0);
-        t.n_mma = (t.ncols + 127) & ~127; t.b_boxes = t.n_mma / 128; t.b_off = rank * (t.n_mma / 2);
-    }
-    return t;
-}
-
-template <int KIND>
-__device__ __forceinline__ void issue_loads2(const TcMaps &maps, const Tile &t, int rank, int kb, uint32_t a_dst,
-                                             uint32_t b_dst, uint32_t bar)
-{
-    if constexpr (KIND == TcUpGate) {
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.xp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
-        const CUtensorMap *bm = rank ? &maps.wup : &maps.wgate;     // gate columns live in CTA 0, up columns in CTA 1
-        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d_pair(b_dst + i * kBoxBytes, bm, bar, kb * 64, t.ho + t.n0 + 64 * i);
-    } else if constexpr (KIND == TcDown) {
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + kb * t.cp + t.m0 + 64 * i);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + kb * 64, t.n0 + t.b_off + 64 * i);
-    } else if constexpr (KIND == TcDownDgrad) {
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.dyp, bar, kb * 64, t.prow0 + t.m0 + 64 * i);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + t.b_off + 64 * i, kb * 64);
-    } else if constexpr (KIND == TcDownWgrad) {
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d_pair(a_dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.hm, bar, 0,
-                             t.pbase + ((t.n0 + t.b_off) / 64 + i) * t.cp + kb * 64);
-    } else if constexpr (KIND == TcUpGateDgrad) {
-        const int half = t.h / 64;
-        const bool second = kb >= half;
-        const int kk = second ? kb - half : kb;
-        const CUtensorMap *am = second ? &maps.db : &maps.da;
-        const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d_pair(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + kk * t.cp + t.m0 + 64 * i);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d_pair(b_dst + i * kBoxBytes, bm, bar, t.n0 + t.b_off + 64 * i, t.ho + kk * 64);
-    } else {
-        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d_pair(a_dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d_pair(b_dst + i * kBoxBytes, &maps.xp, bar, t.n0 + t.b_off + 64 * i, t.prow0 + kb * 64);
-    }
-}
-
-template <int KIND>
-__global__ void __launch_bounds__(kThreads, 1)
-tc_grouped_gemm_pair(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
-{
-    extern __shared__ unsigned char smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
-    unsigned char *smem = smem_raw + pad;
-    const uint32_t stage_base = raw + pad;
-    SmemTail2 *st = reinterpret_cast<SmemTail2 *>(smem + (size_t)kStages2 * kStageBytes2);
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int N = prm.meta.N, d = prm.meta.d;
-    const int rank = (int)cluster_ctarank();
-    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-
-    for (int e = tid; e < N; e += kThreads) {
-        const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
-        const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
-        int mt, nt, nk;
-        expert_shape2<KIND>(cp, h, d, mt, nt, nk);
-        st->ntile[e] = mt * nt;
-        st->key[e] = nk;
-    }
-    if (tid == 0) {
-        for (int s = 0; s < kStages2; ++s) {
-            mbar_init(smem_u32(&st->full[s]), 1);
-            mbar_init(smem_u32(&st->empty[s]), 1);
-        }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&st->tmem_full[a]), 1);
-            mbar_init(smem_u32(&st->tmem_empty[a]), 16);      // 8 epilogue warps of each of the two CTAs
-        }
-        st->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-    for (int e = tid; e < N; e += kThreads) {
-        int rk = 0;
-        const int ke = st->key[e];
-        for (int f = 0; f < N; ++f) {
-            const int kf = st->key[f];
-            rk += (kf > ke) || (kf == ke && f < e);
-        }
-        st->order[rk] = e;
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&st->tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int acc = 0;
-        for (int i = 0; i < N; ++i) { st->tstart[i] = acc; acc += st->ntile[st->order[i]]; }
-        st->tstart[N] = acc;
-    }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                 // both CTAs' barriers exist before any remote arrive or TMA completion
-    tc_fence_after();
-    const uint32_t tmem_base = st->tmem_base;
-    const int total_tiles = st->tstart[N];
-    volatile int *abort_flag = &st->abort_flag;
-
-    if (warp == 0) {
-        // ===================== TMA producer (both CTAs) =====================
-        if (lane == 0) {
-            int stage = 0, cursor = 0;
-            uint32_t phase = 0;
-            long long issued = 0;
-            bool ok = true;
-            for (int rnd = 0, tile = dealt_tile<KIND>(0, cluster_id, n_clusters); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, cluster_id, n_clusters)) {
-                const Tile t = decode_tile2<KIND>(prm, st, tile, cursor, rank);
-                const uint32_t bytes = (uint32_t)(t.a_boxes + t.a_boxes_peer + 2 * t.b_boxes) * kBoxBytes;
-                for (int kb = 0; kb < t.nk; ++kb) {
-                    if (!mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-                    const uint32_t leader_bar = map_to_cta(smem_u32(&st->full[stage]), 0);
-                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&st->full[stage]), bytes);
-                    const uint32_t a_dst = stage_base + stage * kStageBytes2;
-                    issue_loads2<KIND>(maps, t, rank, kb, a_dst, a_dst + kARegion2, leader_bar);
-                    ++issued;
-                    if (++stage == kStages2) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if (!ok && rank == 0) {
-                const int n = issued < kStages2 ? (int)issued : kStages2;
-                for (int i = 1; i <= n; ++i) {
-                    int s = stage - i;
-                    uint32_t ph = phase;
-                    if (s < 0) { s += kStages2; ph ^= 1u; }
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(smem_u32(&st->full[s]), ph) && global_ns() - t0 < kWaitLimitNs) {}
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ===================== MMA issuer (leader CTA only) =====================
-        if (lane == 0 && rank == 0) {
-            int stage = 0, cursor = 0, it = 0;
-            uint32_t phase = 0;
-            bool ok = true;
-            constexpr bool a_mn = KindTraits<KIND>::a_mn, b_mn = KindTraits<KIND>::b_mn;
-            constexpr uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
-            constexpr uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
-            for (int rnd = 0, tile = dealt_tile<KIND>(0, cluster_id, n_clusters); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, cluster_id, n_clusters), ++it) {
-                const Tile t = decode_tile2<KIND>(prm, st, tile, cursor, 0);
-                const int acc = it & 1;
-                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t tacc = tmem_base + (uint32_t)(acc * kAccCols);
-                const uint32_t idesc = make_idesc_pair(a_mn, b_mn, t.n_mma);
-                for (int kb = 0; kb < t.nk; ++kb) {
-                    if (!mbar_wait(smem_u32(&st->full[stage]), phase, abort_flag, prm.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = stage_base + stage * kStageBytes2;
-                    const uint64_t adesc = make_desc(a_addr, a_mn);
-                    const uint64_t bdesc = make_desc(a_addr + kARegion2, b_mn);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_bf16_pair(tacc, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
-                                       (kb > 0 || ks > 0) ? 1u : 0u);
-                    umma_commit_pair(smem_u32(&st->empty[stage]));
-                    if (++stage == kStages2) { stage = 0; phase ^= 1u; }
-                }
-                if (!ok) break;
-                if (t.nk > 0) {
-                    umma_commit_pair(smem_u32(&st->tmem_full[acc]));
-                } else {
-                    mbar_arrive(smem_u32(&st->tmem_full[acc]));
-                    mbar_arrive_cluster(map_to_cta(smem_u32(&st->tmem_full[acc]), 1));
-                }
-            }
-        }
-    } else {
-        // ===================== epilogue (warps 2..9, both CTAs) =====================
-        const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
-        const int row = quad * 32 + lane;
-        int cursor = 0, it = 0;
-        bool ok = true;
-        for (int rnd = 0, tile = dealt_tile<KIND>(0, cluster_id, n_clusters); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, cluster_id, n_clusters), ++it) {
-            const Tile t = decode_tile2<KIND>(prm, st, tile, cursor, rank);
-            const int acc = it & 1;
-            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-            if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, abort_flag, prm.status)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
-            if (t.mrows > 0) {
-                // split the accumulator columns between the two warps of a lane quadrant, store only valid ones
-                const int span = (KIND == TcUpGate) ? t.ncols : t.n_mma;
-                const int chalf = span >> 1;
-                const int c0 = half * chalf, c1 = min((half + 1) * chalf, t.ncols);
-                if (c0 < c1) epilogue_row<KIND>(prm, t, tacc, row, c0, c1, st->epi_stage[warp - 2]);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (rank == 0) mbar_arrive(smem_u32(&st->tmem_empty[acc]));
-                else mbar_arrive_cluster(map_to_cta(smem_u32(&st->tmem_empty[acc]), 0));
-            }
-        }
-    }
-
-    // ---- teardown: nobody leaves while its partner may still touch its shared or tensor memory ----
-    tc_fence_before();
-    __syncthreads();
-    __syncwarp();
-    cluster_sync_all();
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-    }
-}
-
-// ===========================================================================
-// Wide variant: one CTA computes a 256-row tile as two 128-row halves that
-// share the column operand.  A k-block then stages 32 KB of rows + 32 KB of
-// columns for twice the MMA work of the 128-row kernel, i.e. 2/3 of the bytes
-// per FLOP through L2 -> shared memory, which is what bounds the 128-row
-// kernel (it needs ~19.5 TB/s of L2 reads at the MMA rate; the path saturates
-// near 22 TB/s).  The price: both accumulators (2 x 256 TMEM columns) belong
-// to the current tile, so the epilogue of a tile overlaps only the part of the
-// next tile's main loop that does not touch the half being drained.  Used for
-// the products with long K loops, where that exposure is a few percent.
-// ===========================================================================
-constexpr int kStagesW = 3;
-constexpr int kARegionW = 4 * kBoxBytes;            // two halves of 128 rows x 64 K
-constexpr int kStageBytesW = kARegionW + kBRegion;  // 64 KB
-struct SmemTailW {
-    unsigned char epi_stage[8][kEpiWarpBytes];   // one transposing buffer per epilogue warp
-    unsigned long long full[kStagesW], empty[kStagesW], tmem_full[1], tmem_empty[2];
-    unsigned int tmem_base;
-    int abort_flag;
-    int order[kMaxExperts];
-    int key[kMaxExperts];
-    int ntile[kMaxExperts];
-    int tstart[kMaxExperts + 1];
-};
-constexpr size_t kSmemBytesW = 1024 + (size_t)kStagesW * kStageBytesW + sizeof(SmemTailW);
-
-template <int KIND>
-__device__ __forceinline__ void expert_shape_wide(int cp, int h, int d, int &mt, int &nt, int &nk)
-{
-    if constexpr (KIND == TcUpGate)      { mt = (cp + 255) / 256; nt = (h + 127) / 128; nk = d / 64; }
-    if constexpr (KIND == TcDown)        { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = h / 64; }
-    if constexpr (KIND == TcDownDgrad)   { mt = (cp + 255) / 256; nt = (h + 255) / 256; nk = d / 64; }
-    if constexpr (KIND == TcDownWgrad)   { mt = (d + 255) / 256;  nt = (h + 255) / 256; nk = cp / 64; }
-    if constexpr (KIND == TcUpGateDgrad) { mt = (cp + 255) / 256; nt = (d + 255) / 256; nk = 2 * (h / 64); }
-    if constexpr (KIND == TcUpGateWgrad) { mt = 2 * ((h + 255) / 256); nt = (d + 255) / 256; nk = cp / 64; }
-}
-
-// First half (rows m0 .. m0+127) of wide tile `tile`; a_boxes_peer carries the second half's boxes.
-template <int KIND>
-__device__ __forceinline__ Tile decode_tile_wide(const TcParams &prm, const SmemTailW *st, int tile, int &cursor)
-{
-    const int N = prm.meta.N, d = prm.meta.d;
-    while (cursor + 1 < N && tile >= st->tstart[cursor + 1]) ++cursor;
-    Tile t;
-    t.e = st->order[cursor];
-    t.ho = prm.meta.hoff[t.e];
-    t.h = prm.meta.hoff[t.e + 1] - t.ho;
-    t.prow0 = prm.poffsets[t.e];
-    t.cp = prm.poffsets[t.e + 1] - t.prow0;
-    t.pbase = (int)(prm.ebase[t.e] >> 6);
-    int mt, nt, nk;
-    expert_shape_wide<KIND>(t.cp, t.h, d, mt, nt, nk);
-    const int local = tile - st->tstart[cursor];
-    constexpr bool n_fastest = (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad);
-    int mb, nb;
-    tile_coords<n_fastest>(local, mt, nt, group_row_tiles(d, 256), mb, nb);
-    t.nk = nk;
-    t.which = 0;
-    int row_extent;
-    if constexpr (KIND == TcDownWgrad) row_extent = d;
-    else if constexpr (KIND == TcUpGateWgrad) { row_extent = t.h; t.which = mb & 1; mb >>= 1; }
-    else row_extent = t.cp;
-    t.m0 = mb * 256;
-    t.mrows = max(0, min(128, row_extent - t.m0));
-    t.a_boxes = t.mrows / 64;
-    t.a_boxes_peer = max(0, min(128, row_extent - t.m0 - 128)) / 64;
-    t.b_off = 0;
-    if constexpr (KIND == TcUpGate) {
-        t.n0 = nb * 128; t.ncols = min(128, t.h - t.n0);
-        t.n_mma = 2 * t.ncols; t.b_boxes = t.n_mma / 64;
-    } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad || KIND == TcUpGateWgrad) {
-        t.n0 = nb * 256; t.ncols = min(256, d - t.n0);
-        t.n_mma = t.ncols; t.b_boxes = t.ncols / 64;
-    } else {
-        t.n0 = nb * 256; t.ncols = min(256, t.h - t.n0);
-        t.n_mma = t.ncols; t.b_boxes = t.ncols / 64;
-    }
-    return t;
-}
-
-__device__ __forceinline__ Tile second_half(const Tile &t)
-{
-    Tile u = t;
-    u.m0 = t.m0 + 128;
-    u.a_boxes = t.a_boxes_peer;
-    u.mrows = 64 * t.a_boxes_peer;
-    return u;
-}
-
-// Row-operand boxes of one 128-row half.
-template <int KIND>
-__device__ __forceinline__ void load_rows(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
-{
-    if constexpr (KIND == TcUpGate) {
-        tma_load_rows(dst, &maps.xp, &maps.xp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
-    } else if constexpr (KIND == TcDown) {
-        tma_load_rows(dst, &maps.hm, &maps.hm128, bar, 0, t.pbase + kb * t.cp + t.m0, t.a_boxes);
-    } else if constexpr (KIND == TcDownDgrad) {
-        tma_load_rows(dst, &maps.dyp, &maps.dyp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
-    } else if constexpr (KIND == TcDownWgrad) {
-        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
-    } else if constexpr (KIND == TcUpGateDgrad) {
-        const int half = t.h / 64;
-        const bool second = kb >= half;
-        const int kk = second ? kb - half : kb;
-        tma_load_rows(dst, second ? &maps.db : &maps.da, second ? &maps.db128 : &maps.da128, bar, 0,
-                      t.pbase + kk * t.cp + t.m0, t.a_boxes);
-    } else {
-        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
-        for (int i = 0; i < t.a_boxes; ++i)
-            tma_load_2d(dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
-    }
-}
-
-// Column-operand boxes of a tile.
-template <int KIND>
-__device__ __forceinline__ void load_cols(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
-{
-    if constexpr (KIND == TcUpGate) {
-        const int nb = t.ncols / 64;
-        tma_load_rows(dst, &maps.wgate, &maps.wgate128, bar, kb * 64, t.ho + t.n0, nb);
-        tma_load_rows(dst + nb * kBoxBytes, &maps.wup, &maps.wup128, bar, kb * 64, t.ho + t.n0, nb);
-    } else if constexpr (KIND == TcDown) {
-        tma_load_rows(dst, &maps.wdown, &maps.wdown128, bar, t.ho + kb * 64, t.n0, t.b_boxes);
-    } else if constexpr (KIND == TcDownDgrad) {
-        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + 64 * i, kb * 64);
-    } else if constexpr (KIND == TcDownWgrad) {
-        for (int i = 0; i < t.b_boxes; ++i)
-            tma_load_2d(dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + (t.n0 / 64 + i) * t.cp + kb * 64);
-    } else if constexpr (KIND == TcUpGateDgrad) {
-        const int half = t.h / 64;
-        const bool second = kb >= half;
-        const int kk = second ? kb - half : kb;
-        const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
-        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, bm, bar, t.n0 + 64 * i, t.ho + kk * 64);
-    } else {
-        for (int i = 0; i < t.b_boxes; ++i) tma_load_2d(dst + i * kBoxBytes, &maps.xp, bar, t.n0 + 64 * i, t.prow0 + kb * 64);
-    }
-}
-
-template <int KIND>
-__global__ void __launch_bounds__(kThreads, 1)
-tc_grouped_gemm_wide(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
-{
-    extern __shared__ unsigned char smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
-    unsigned char *smem = smem_raw + pad;
-    const uint32_t stage_base = raw + pad;
-    SmemTailW *st = reinterpret_cast<SmemTailW *>(smem + (size_t)kStagesW * kStageBytesW);
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int N = prm.meta.N, d = prm.meta.d;
-
-    for (int e = tid; e < N; e += kThreads) {
-        const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
-        const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
-        int mt, nt, nk;
-        expert_shape_wide<KIND>(cp, h, d, mt, nt, nk);
-        st->ntile[e] = mt * nt;
-        st->key[e] = nk;
-    }
-    if (tid == 0) {
-        for (int s = 0; s < kStagesW; ++s) {
-            mbar_init(smem_u32(&st->full[s]), 1);
-            mbar_init(smem_u32(&st->empty[s]), 1);
-        }
-        mbar_init(smem_u32(&st->tmem_full[0]), 1);
-        mbar_init(smem_u32(&st->tmem_empty[0]), 256);
-        mbar_init(smem_u32(&st->tmem_empty[1]), 256);
-        st->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    __syncthreads();
-    for (int e = tid; e < N; e += kThreads) {
-        int rk = 0;
-        const int ke = st->key[e];
-        for (int f = 0; f < N; ++f) {
-            const int kf = st->key[f];
-            rk += (kf > ke) || (kf == ke && f < e);
-        }
-        st->order[rk] = e;
-    }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&st->tmem_base)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    __syncthreads();
-    if (tid == 0) {
-        int acc = 0;
-        for (int i = 0; i < N; ++i) { st->tstart[i] = acc; acc += st->ntile[st->order[i]]; }
-        st->tstart[N] = acc;
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = st->tmem_base;
-    const int total_tiles = st->tstart[N];
-    volatile int *abort_flag = &st->abort_flag;
-
-    if (warp == 0) {
-        // ===================== TMA producer =====================
-        if (lane == 0) {
-            int stage = 0, cursor = 0;
-            uint32_t phase = 0;
-            long long issued = 0;
-            bool ok = true;
-            for (int rnd = 0, tile = dealt_tile<KIND>(0, blockIdx.x, gridDim.x); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, blockIdx.x, gridDim.x)) {
-                const Tile t0 = decode_tile_wide<KIND>(prm, st, tile, cursor);
-                const Tile t1 = second_half(t0);
-                const uint32_t bytes = (uint32_t)(t0.a_boxes + t1.a_boxes + t0.b_boxes) * kBoxBytes;
-                for (int kb = 0; kb < t0.nk; ++kb) {
-                    if (!mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-                    const uint32_t bar = smem_u32(&st->full[stage]);
-                    mbar_arrive_expect_tx(bar, bytes);
-                    const uint32_t a_dst = stage_base + stage * kStageBytesW;
-                    load_rows<KIND>(maps, t0, kb, a_dst, bar);
-                    load_rows<KIND>(maps, t1, kb, a_dst + kARegion, bar);
-                    load_cols<KIND>(maps, t0, kb, a_dst + kARegionW, bar);
-                    ++issued;
-                    if (++stage == kStagesW) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if (!ok) {
-                const int n = issued < kStagesW ? (int)issued : kStagesW;
-                for (int i = 1; i <= n; ++i) {
-                    int s = stage - i;
-                    uint32_t ph = phase;
-                    if (s < 0) { s += kStagesW; ph ^= 1u; }
-                    const unsigned long long tb = global_ns();
-                    while (!mbar_try_wait(smem_u32(&st->full[s]), ph) && global_ns() - tb < kWaitLimitNs) {}
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ===================== MMA issuer =====================
-        if (lane == 0) {
-            int stage = 0, cursor = 0;
-            uint32_t phase = 0;
-            uint32_t use0 = 0, use1 = 0;         // how often each accumulator has been handed to the epilogue
-            bool ok = true;
-            constexpr bool a_mn = KindTraits<KIND>::a_mn, b_mn = KindTraits<KIND>::b_mn;
-            constexpr uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
-            constexpr uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
-            for (int rnd = 0, tile = dealt_tile<KIND>(0, blockIdx.x, gridDim.x); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, blockIdx.x, gridDim.x)) {
-                const Tile t = decode_tile_wide<KIND>(prm, st, tile, cursor);
-                const bool two = t.a_boxes_peer > 0;
-                if (!mbar_wait(smem_u32(&st->tmem_empty[0]), (use0 & 1u) ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t idesc = make_idesc(a_mn, b_mn, t.n_mma);
-                for (int kb = 0; kb < t.nk; ++kb) {
-                    if (!mbar_wait(smem_u32(&st->full[stage]), phase, abort_flag, prm.status)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = stage_base + stage * kStageBytesW;
-                    const uint64_t adesc0 = make_desc(a_addr, a_mn);
-                    const uint64_t adesc1 = make_desc(a_addr + kARegion, a_mn);
-                    const uint64_t bdesc = make_desc(a_addr + kARegionW, b_mn);
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        umma_bf16(tmem_base, adesc0 + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
-                                  (kb > 0 || ks > 0) ? 1u : 0u);
-                    if (two) {
-                        if (kb == 0) {
-                            // the second accumulator may still be draining: the first half's MMAs above are already queued
-                            if (!mbar_wait(smem_u32(&st->tmem_empty[1]), (use1 & 1u) ^ 1u, abort_flag, prm.status)) { ok = false; break; }
-                            tc_fence_after();
-                        }
-#pragma unroll
-                        for (int ks = 0; ks < 4; ++ks)
-                            umma_bf16(tmem_base + kAccCols, adesc1 + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step),
-                                      idesc, (kb > 0 || ks > 0) ? 1u : 0u);
-                    }
-                    umma_commit(smem_u32(&st->empty[stage]));
-                    if (++stage == kStagesW) { stage = 0; phase ^= 1u; }
-                }
-                if (!ok) break;
-                if (t.nk > 0) umma_commit(smem_u32(&st->tmem_full[0]));
-                else mbar_arrive(smem_u32(&st->tmem_full[0]));
-                ++use0;
-                if (two) ++use1;
-            }
-        }
-    } else {
-        // ===================== epilogue (warps 2..9) =====================
-        const int quad = warp & 3;
-        const int half = (warp - 2) >> 2;
-        const int row = quad * 32 + lane;
-        int cursor = 0, it = 0;
-        bool ok = true;
-        for (int rnd = 0, tile = dealt_tile<KIND>(0, blockIdx.x, gridDim.x); tile < total_tiles && ok;
-                 tile = dealt_tile<KIND>(++rnd, blockIdx.x, gridDim.x), ++it) {
-            const Tile t0 = decode_tile_wide<KIND>(prm, st, tile, cursor);
-            if (!mbar_wait(smem_u32(&st->tmem_full[0]), (uint32_t)it & 1u, abort_flag, prm.status)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16);
-            const int chalf = t0.ncols >> 1;
-            epilogue_row<KIND>(prm, t0, tacc, row, half * chalf, (half + 1) * chalf, st->epi_stage[warp - 2]);
-            tc_fence_before();
-            mbar_arrive(smem_u32(&st->tmem_empty[0]));
-            if (t0.a_boxes_peer > 0) {
-                const Tile t1 = second_half(t0);
-                epilogue_row<KIND>(prm, t1, tacc + kAccCols, row, half * chalf, (half + 1) * chalf,
-                                   st->epi_stage[warp - 2]);
-                tc_fence_before();
-                mbar_arrive(smem_u32(&st->tmem_empty[1]));
-            }
-        }
-    }
-
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        __syncwarp();
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-    }
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= Ttok * m.k) return;
+    const int e = topk_idx[i], prow = prow_of[i];
+    if (e < 0 || e >= m.N || prow < 0 || prow >= Pmax) { atomicMax(status, kDevBounds); return; }
+    const int slots = 2 * ((m.hoff[e + 1] - m.hoff[e] + 255) / 256);     // two per 256-column tile
+    float acc = 0.f;
+    for (int sl = 0; sl < slots; ++sl) acc += dg_part[(size_t)sl * Pmax + prow];
+    const float g = topk_gate[i];
+    dg[i] = (g > 0.f) ? acc / g : 0.f;
 }
 
 // ---------------------------------------------------------------------------
@@ -1484,24 +1168,25 @@ EncodeTiledFn get_encode()
     return fn;
 }
 
-// bf16 row-major matrix [rows, cols] seen as a 2-D tensor, boxes of 64 columns x box_rows rows, 128-byte swizzle.
-bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows = 64)
+// bf16 row-major matrix [rows, cols] seen as a 2-D tensor, boxes of box_cols columns x box_rows rows.
+bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows = 64,
+               uint32_t box_cols = 64, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B)
 {
     EncodeTiledFn fn = get_encode();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {cols * 2};
-    const cuuint32_t box[2] = {64, box_rows};
+    const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
 
 bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
-                  bool backward)
+                  const void *x, bool backward)
 {
     const uint64_t panel_rows = L.hb / 64;
     bool ok = true;
@@ -1513,6 +1198,7 @@ bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsP
     both(&maps.wup, &maps.wup128, w->w_up, m.S, m.d);
     both(&maps.wdown, &maps.wdown128, w->w_down, m.d, m.S);
     both(&maps.hm, &maps.hm128, p.hm, panel_rows, 64);
+    ok = ok && encode_2d(&maps.xg, x, (uint64_t)L.T, m.d, 1);
     if (backward) {
         both(&maps.dyp, &maps.dyp128, p.dyp, L.Pmax, m.d);
         both(&maps.da, &maps.da128, p.da, panel_rows, 64);
@@ -1527,90 +1213,37 @@ bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsP
 
 namespace {
 
-TcParams make_params(const LayerMeta &m, const WsPtrs &p, const modse_wgrads_t *g, bool save, bool out_f32)
+template <int KIND, bool WIDE, int VAR>
+cudaError_t launch_one(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
 {
-    TcParams prm{};
-    prm.meta = m;
-    prm.poffsets = p.poffsets;
-    prm.ebase = p.ebase;
-    prm.status = p.status;
-    prm.pgate = p.pgate;
-    prm.hm = (__nv_bfloat16 *)p.hm;
-    prm.sp = (__nv_bfloat16 *)p.a_pre;
-    prm.sq = (__nv_bfloat16 *)p.b_pre;
-    prm.da = (__nv_bfloat16 *)p.da;
-    prm.db = (__nv_bfloat16 *)p.db;
-    prm.o = (float *)p.o;
-    prm.dxp = (float *)p.dxp;
-    if (g) {
-        prm.dw_gate = (__nv_bfloat16 *)g->dw_gate;
-        prm.dw_up = (__nv_bfloat16 *)g->dw_up;
-        prm.dw_down = (__nv_bfloat16 *)g->dw_down;
-    }
-    prm.save = save ? 1 : 0;
-    prm.out_f32 = out_f32 ? 1 : 0;
-    return prm;
-}
-
-// Launches the two-CTA kernel with as many clusters as can be resident at once (tiles are dealt
-// statically, so a cluster that is not resident would hold its share back).
-template <int KIND>
-cudaError_t launch_kind_pair(const TcMaps &maps, const TcParams &prm, int sms, cudaStream_t s, int *launches)
-{
-    auto kern = tc_grouped_gemm_pair<KIND>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes2);
+    auto kern = tc_grouped_gemm<KIND, WIDE, VAR>;
+    constexpr size_t smem = smem_bytes<WIDE>();
+    // the shared-memory attribute of a kernel is set once per process and device
+    static unsigned long long attr_done = 0;      // bit per device ordinal (devices beyond 63 set it every time)
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(sms & ~1));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kSmemBytes2;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    static int max_clusters[6] = {0, 0, 0, 0, 0, 0};
-    if (max_clusters[KIND] == 0) {
-        int n = 0;
-        e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+    if (dev < 0 || dev > 63 || !((attr_done >> dev) & 1ull)) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        if (n < 1) return cudaErrorInvalidConfiguration;
-        max_clusters[KIND] = n;
+        if (dev >= 0 && dev <= 63) attr_done |= 1ull << dev;
     }
-    const int clusters = max_clusters[KIND] < sms / 2 ? max_clusters[KIND] : sms / 2;
-    cfg.gridDim = dim3((unsigned)(2 * clusters));
-    e = cudaLaunchKernelEx(&cfg, kern, maps, prm);
-    if (e == cudaSuccess && launches) ++*launches;
-    return e;
-}
-
-template <int KIND>
-cudaError_t launch_kind_wide(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
-{
-    auto kern = tc_grouped_gemm_wide<KIND>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytesW);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytesW, s>>>(maps, prm);
+    kern<<<grid, kThreads, smem, s>>>(maps, prm);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }
 
-template <int KIND>
-cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, int mask, cudaStream_t s, int *launches)
+template <int KIND, bool HAS_VAR>
+cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, bool wide, int var, cudaStream_t s, int *launches)
 {
-    if ((mask >> 8) & (1 << KIND)) return launch_kind_wide<KIND>(maps, prm, grid, s, launches);
-    if (mask & (1 << KIND)) return launch_kind_pair<KIND>(maps, prm, grid, s, launches);
-    auto kern = tc_grouped_gemm<KIND>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytes, s>>>(maps, prm);
-    e = cudaGetLastError();
-    if (e == cudaSuccess && launches) ++*launches;
-    return e;
+    if constexpr (HAS_VAR) {
+        if (var)
+            return wide ? launch_one<KIND, true, 1>(maps, prm, grid, s, launches)
+                        : launch_one<KIND, false, 1>(maps, prm, grid, s, launches);
+    }
+    return wide ? launch_one<KIND, true, 0>(maps, prm, grid, s, launches)
+                : launch_one<KIND, false, 0>(maps, prm, grid, s, launches);
 }
 
 int sm_count(TcPlan &plan)
@@ -1628,21 +1261,60 @@ int sm_count(TcPlan &plan)
 
 }  // namespace
 
-cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const LayerMeta &m, const WsPtrs &p,
-                      const modse_wgrads_t *g, bool save, bool out_f32, cudaStream_t s, int *launches)
+cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const LayerMeta &m, const WsLayout &L,
+                      const WsPtrs &p, const modse_wgrads_t *g, bool save, bool out_f32, int fuse, float *scatter_out,
+                      cudaStream_t s, int *launches)
 {
-    const TcParams prm = make_params(m, p, g, save, out_f32);
-    const int grid = sm_count(plan);
-    const int mask = plan.tile_mask >= 0 ? plan.tile_mask : tc_pair_mask();
-    switch (kind) {
-    case TcUpGate: return launch_kind<TcUpGate>(maps, prm, grid, mask, s, launches);
-    case TcDown: return launch_kind<TcDown>(maps, prm, grid, mask, s, launches);
-    case TcDownDgrad: return launch_kind<TcDownDgrad>(maps, prm, grid, mask, s, launches);
-    case TcDownWgrad: return launch_kind<TcDownWgrad>(maps, prm, grid, mask, s, launches);
-    case TcUpGateDgrad: return launch_kind<TcUpGateDgrad>(maps, prm, grid, mask, s, launches);
-    case TcUpGateWgrad: return launch_kind<TcUpGateWgrad>(maps, prm, grid, mask, s, launches);
+    TcParams prm{};
+    prm.meta = m;
+    prm.poffsets = p.poffsets;
+    prm.ebase = p.ebase;
+    prm.status = p.status;
+    prm.tile_counter = p.status + 4 + (int)kind;
+    prm.pgate = p.pgate;
+    prm.ptoken_of = p.ptoken_of;
+    prm.hm = (__nv_bfloat16 *)p.hm;
+    prm.sp = (__nv_bfloat16 *)p.a_pre;
+    prm.sq = (__nv_bfloat16 *)p.b_pre;
+    prm.da = (__nv_bfloat16 *)p.da;
+    prm.db = (__nv_bfloat16 *)p.db;
+    prm.o = (float *)p.o;
+    prm.dxp = (float *)p.dxp;
+    prm.dg_part = p.dg_part;
+    prm.scatter_out = scatter_out;
+    if (g) {
+        prm.dw_gate = (__nv_bfloat16 *)g->dw_gate;
+        prm.dw_up = (__nv_bfloat16 *)g->dw_up;
+        prm.dw_down = (__nv_bfloat16 *)g->dw_down;
     }
-    return cudaErrorInvalidValue;
+    prm.wait_limit_ns = (unsigned long long)g_wait_limit_ms * 1000000ull;
+    prm.Pmax = L.Pmax;
+    prm.T = L.T;
+    prm.save = save ? 1 : 0;
+    prm.out_f32 = out_f32 ? 1 : 0;
+    prm.dynamic = g_dynamic_tiles;
+    prm.skip_tile = (g_skip_kind == (int)kind) ? g_skip_tile : -1;
+    const int grid = sm_count(plan);
+    const int mask = plan.tile_mask >= 0 ? plan.tile_mask : tc_default_plan();
+    const bool wide = ((mask >> (int)kind) & 1) != 0;
+    cudaError_t e = cudaErrorInvalidValue;
+    switch (kind) {
+    case TcUpGate: e = launch_kind<TcUpGate, true>(maps, prm, grid, wide, fuse & kFuseGather, s, launches); break;
+    case TcDown: e = launch_kind<TcDown, true>(maps, prm, grid, wide, fuse & kFuseScatter, s, launches); break;
+    case TcDownDgrad: e = launch_kind<TcDownDgrad, true>(maps, prm, grid, wide, fuse & kFuseDgRowdot, s, launches); break;
+    case TcDownWgrad: e = launch_kind<TcDownWgrad, false>(maps, prm, grid, wide, 0, s, launches); break;
+    case TcUpGateDgrad: e = launch_kind<TcUpGateDgrad, true>(maps, prm, grid, wide, fuse & kFuseScatter, s, launches); break;
+    case TcUpGateWgrad: e = launch_kind<TcUpGateWgrad, false>(maps, prm, grid, wide, 0, s, launches); break;
+    }
+    if (e != cudaSuccess) return e;
+    if (kind == TcDownDgrad && (fuse & kFuseDgRowdot)) {
+        const int n = L.T * m.k;
+        dg_finish_kernel<<<(n + 255) / 256, 256, 0, s>>>(m, L.T, L.Pmax, p.topk_idx, p.topk_gate, p.prow_of, p.dg_part, p.dg,
+                                                         p.status);
+        e = cudaGetLastError();
+        if (e == cudaSuccess && launches) ++*launches;
+    }
+    return e;
 }
 
 }  // namespace modse

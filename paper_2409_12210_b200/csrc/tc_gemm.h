@@ -7,21 +7,6 @@
 
 namespace modse {
 
-// Host-side state owned by a layer object.
-struct TcPlan {
-    int sm_count = 0;   // number of SMs of the device the layer last ran on
-    int tile_mask = -1; // which kernel variant runs each product (layout of tc_pair_mask()); -1: the process-wide default
-};
-
-// Process-wide debugging switch: run bf16 layers through the fp32-FMA grouped
-// GEMMs instead of the tensor-core kernels.
-bool tc_force_simt();
-void tc_set_force_simt(int on);
-
-// Which of the six products run on the two-CTA (cta_group::2) kernel: bit k = kind k.
-void tc_set_pair_mask(int mask);
-int tc_pair_mask();
-
 // The six grouped products of the layer (Sec. 3.1, Eq. 4 and its gradient).
 enum TcKind : int {
     TcUpGate = 0,       // Hm = g * silu(xp Wg^T) * (xp Wu^T), optionally saving B*silu'(A) and silu(A)
@@ -32,17 +17,63 @@ enum TcKind : int {
     TcUpGateWgrad = 5   // dWg = dA^T xp, dWu = dB^T xp
 };
 
-// Tensor maps of every TMA-loaded buffer (bf16, 64 x 64 boxes, 128-byte swizzle), and the same tensors
-// with boxes of 128 rows: where an operand's rows are contiguous (K-major operands), one 16 KB copy fills
-// what two 8 KB copies would, in the same shared-memory layout, and the larger copies measured faster.
+// Tile plan: bit k set = product kind k runs on 256-row tiles (two 128-row halves that share the column
+// operand), clear = on 128-row tiles with two accumulators in flight.  Default: the four products with
+// long K loops (down, down wgrad, up/gate dgrad, up/gate wgrad) on 256-row tiles.
+constexpr int kTcDefaultPlan = (1 << TcDown) | (1 << TcDownWgrad) | (1 << TcUpGateDgrad) | (1 << TcUpGateWgrad);
+constexpr int kTcPlanBits = 63;
+
+// Optional fusions across the permutation (what lies either side of the permute / un-permute steps).
+enum : int {
+    kFuseGather = 1,    // up/gate product gathers its rows from x through the permutation (TMA gather), not from xp
+    kFuseDgRowdot = 2,  // dg = rowdot(dyp Wd, Hm) / g inside the down-dgrad epilogue; o is not read in backward
+    kFuseScatter = 4,   // down and up/gate dgrad add their rows straight into fp32 y / dx (k <= 2, fp32 outputs)
+    kFuseAll = 7
+};
+
+// Tensor maps of every TMA-accessed buffer.
+//   loads : bf16, boxes of 64 columns x 64 rows with the 128-byte swizzle, and the same tensors with boxes of
+//           128 rows (where an operand's rows are contiguous one 16 KB copy fills what two 8 KB copies would);
+//   xg    : x [T, d] with boxes one row high, for the row-gathering load of the fused up/gate product.
 struct TcMaps {
     CUtensorMap xp, dyp, wgate, wup, wdown, hm, da, db;
     CUtensorMap xp128, dyp128, wgate128, wup128, wdown128, hm128, da128, db128;
+    CUtensorMap xg;
 };
 
+// What the maps were encoded for; a call whose key matches reuses them.
+struct TcMapKey {
+    const void *ws = nullptr, *x = nullptr, *w_gate = nullptr, *w_up = nullptr, *w_down = nullptr;
+    int T = -1, backward = -1;
+    bool operator==(const TcMapKey &o) const
+    {
+        return ws == o.ws && x == o.x && w_gate == o.w_gate && w_up == o.w_up && w_down == o.w_down && T == o.T &&
+               backward == o.backward;
+    }
+};
+
+// Host-side state owned by a layer object.
+struct TcPlan {
+    int sm_count = 0;    // number of SMs of the device the layer last ran on
+    int tile_mask = -1;  // tile plan (bit per product, see above); -1: the process-wide default
+    TcMaps maps_fwd, maps_bwd;
+    TcMapKey key_fwd, key_bwd;
+};
+
+// Process-wide debugging switches.
+bool tc_force_simt();                 // run bf16 layers through the fp32-FMA grouped GEMMs
+void tc_set_force_simt(int on);
+void tc_set_default_plan(int mask);   // tile plan used by layers that have none of their own
+int tc_default_plan();
+void tc_set_dynamic_tiles(int on);    // 1 (default): CTAs take tiles from a shared counter; 0: tiles are dealt statically
+void tc_set_wait_limit_ms(int ms);    // limit of every bounded wait inside the kernels (default 2000)
+void tc_set_skip_tile(int kind, int tile);   // the producer of the CTA that gets `tile` of product `kind` stops there (-1: off)
+
 bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
-                  bool backward);
-cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const LayerMeta &m, const WsPtrs &p,
-                      const modse_wgrads_t *g, bool save, bool out_f32, cudaStream_t s, int *launches);
+                  const void *x, bool backward);
+// fuse: the kFuse* bits that apply to this product
+cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const LayerMeta &m, const WsLayout &L,
+                      const WsPtrs &p, const modse_wgrads_t *g, bool save, bool out_f32, int fuse, float *scatter_out,
+                      cudaStream_t s, int *launches);
 
 }  // namespace modse

@@ -107,12 +107,34 @@ def test_noise_gate_argument_errors_need_no_gpu():
 def test_tile_plan_validation_needs_no_gpu():
     layer = B.ModseLayer(2048, [2816, 8448], 2)
     assert layer.tile_plan() == -1                      # library default until tuned or set
-    layer.set_tile_plan(0x3A00)
-    assert layer.tile_plan() == 0x3A00
+    layer.set_tile_plan(B.DEFAULT_TILE_PLAN)
+    assert layer.tile_plan() == B.DEFAULT_TILE_PLAN
     layer.set_tile_plan(-1)
     assert layer.tile_plan() == -1
-    for bad in (-2, 0x4000, 0x40):
+    for bad in (-2, 0x100, 0x40):
         with pytest.raises(B.ModseError) as ei:
             layer.set_tile_plan(bad)
         assert ei.value.status == B.MODSE_ERR_INVALID_ARG
     layer.destroy()
+
+
+def test_fusion_flags_and_debug_switches_need_no_gpu():
+    layer = B.ModseLayer(2048, [2816, 8448], 2)
+    assert layer.fusion() == 0
+    layer.set_fusion(B.MODSE_FUSE_GATHER | B.MODSE_FUSE_DG_ROWDOT | B.MODSE_FUSE_SCATTER)
+    assert layer.fusion() == 7
+    with pytest.raises(B.ModseError) as ei:
+        layer.set_fusion(8)
+    assert ei.value.status == B.MODSE_ERR_INVALID_ARG
+    layer.set_debug_checks(True)
+    prow, guard, pmax = layer.debug_workspace_offsets(B.MODSE_BF16, 1000, True)
+    assert prow % 256 == 0 and guard % 256 == 0 and pmax % 128 == 0 and pmax >= 2000
+    # the guard blocks are part of the workspace in either mode
+    n = layer.workspace_bytes(B.MODSE_BF16, 1000, True)
+    layer.set_debug_checks(False)
+    assert layer.workspace_bytes(B.MODSE_BF16, 1000, True) == n
+    layer.destroy()
+    B.debug_set_wait_limit_ms(2000)
+    B.debug_skip_tile_loads(-1, -1)
+    B.debug_set_dynamic_tiles(True)
+    B.debug_set_default_tile_plan(B.DEFAULT_TILE_PLAN)

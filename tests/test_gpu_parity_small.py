@@ -1,9 +1,10 @@
 """GPU parity: the CUDA library through its C ABI against the fp64 oracle,
 element by element, at sizes the oracle finishes in seconds.
 
-Tolerances: routing tables bit-exact, gates 5e-6 absolute (fp32 logits summed over up to
-2048 products on tensor cores: measured 1.4e-6 at d = 2048), every floating
-tensor max|err|/RMS(ref) <= 1e-4 for the fp32 type and <= 2e-2 for bf16."""
+Tolerances: routing tables bit-exact, gates within the per-token bound helpers.gate_tolerance
+derives from the router's order of additions, every floating tensor max|err|/RMS(ref) <= 1e-4
+for the fp32 type and <= 2e-2 for bf16; the expert weight gradients are held to that bound
+expert by expert (each expert's gradient normalised by its own RMS)."""
 import dataclasses
 
 import numpy as np
@@ -137,6 +138,7 @@ def test_bf16_degenerate_and_ragged_shapes(T, k, widths, d):
     # dz = g (dg - sum g dg) cancels; over one or two tokens its RMS is that of a few numbers,
     # so dz and dW_router = dz^T x keep the max bound above and are left out of the RMS one
     H.check_rms(gpu, ora, RMS_TOL_BF16, skip=("dz", "dw_router") if T < 64 else ())
+    H.check_wgrads_per_expert(inp, gpu, ora, TOL_BF16)
 
 
 def test_bf16_single_expert_top1_is_a_dense_swiglu_ffn():
@@ -158,6 +160,9 @@ def test_bf16_empty_expert_gets_zero_weight_gradients():
     # the pooled max bound is kept for the token-major tensors, the RMS bound for all
     H.check_all(inp, gpu, ora, TOL_BF16, only=("y", "dx", "dg", "dz", "dw_router"))
     H.check_rms(gpu, ora, RMS_TOL_BF16)
+    # all-positive tokens share a large common component, which makes single hidden units' gradient rows many
+    # times larger than the tensor's RMS: expert by expert the max bound is held at twice its value here
+    H.check_wgrads_per_expert(inp, gpu, ora, 2 * TOL_BF16)
     h0, h1 = sum(SMALL_BF16.ffn_sizes[:2]), sum(SMALL_BF16.ffn_sizes[:3])
     assert np.all(gpu["dw_gate"][h0:h1] == 0) and np.all(gpu["dw_up"][h0:h1] == 0)
     assert np.all(gpu["dw_down"][:, h0:h1] == 0)
@@ -166,33 +171,45 @@ def test_bf16_empty_expert_gets_zero_weight_gradients():
 @pytest.mark.parametrize("n_experts", [16, 40, 256])
 def test_bf16_many_experts(n_experts):
     # 16 experts: two 8-expert tiles in the tensor-core router; 40: the general fp32-FMA router;
-    # 256: the largest number of experts the library accepts (about 23 assignments per expert)
+    # 256: the largest number of experts the library accepts (about 94 assignments per expert: every group is
+    # one ragged 128-row tile, some above and some below the token count from which the max bound is asserted)
     rng = np.random.default_rng(n_experts)
     widths = tuple(int(w) for w in rng.choice([64, 128, 192, 256], n_experts))
-    cfg = I.LayerConfig(f"bf16_N{n_experts}", "bf16", 256, widths, 2, 3000, seed=n_experts, weight_std=0.05)
+    n_tokens = 3000 if n_experts < 256 else 12000
+    cfg = I.LayerConfig(f"bf16_N{n_experts}", "bf16", 256, widths, 2, n_tokens, seed=n_experts, weight_std=0.05)
     inp, _ = H.screened(cfg)
     gpu = H.run_gpu(inp, True, out_f32=True)
     ora = H.run_oracle(inp, True)
     H.check_all(inp, gpu, ora, TOL_BF16, only=("y", "dx", "dg", "dz", "dw_router"))
     H.check_rms(gpu, ora, RMS_TOL_BF16)
+    # expert by expert, against each expert's own RMS: a wrong tile tail in one expert of many cannot hide
+    # in a pooled figure (experts with few tokens: see helpers.check_wgrads_per_expert).
+    worst = H.check_wgrads_per_expert(inp, gpu, ora, TOL_BF16)
+    print(f"N = {n_experts}: worst per-expert weight-gradient errors {worst}, counts "
+          f"{int(ora['rt'].counts.min())}..{int(ora['rt'].counts.max())}")
 
 
-def test_bf16_results_are_bitwise_reproducible_and_independent_of_tile_shape():
+def test_bf16_results_are_bitwise_reproducible_and_independent_of_tile_shape_and_tile_order():
     from paper_2409_12210_b200 import binding as B
     inp, _ = H.screened(SMALL_BF16)
     a = H.run_gpu(inp, True)
     b = H.run_gpu(inp, True)
-    B.debug_set_pair_kernels(0)                     # 128-row tiles everywhere
     try:
+        B.debug_set_default_tile_plan(0)               # 128-row tiles everywhere
         c = H.run_gpu(inp, True)
-        B.debug_set_pair_kernels(63)                # two-SM tiles everywhere
+        B.debug_set_default_tile_plan(63)              # 256-row tiles everywhere
         e = H.run_gpu(inp, True)
+        B.debug_set_default_tile_plan(B.DEFAULT_TILE_PLAN)
+        B.debug_set_dynamic_tiles(False)               # tiles dealt round-robin instead of taken from the counter
+        f = H.run_gpu(inp, True)
     finally:
-        B.debug_set_pair_kernels((2 | 8 | 16 | 32) << 8)   # the library's default
+        B.debug_set_default_tile_plan(B.DEFAULT_TILE_PLAN)
+        B.debug_set_dynamic_tiles(True)
     for k in ("y", "dx", "dw_router", "dw_gate", "dw_up", "dw_down", "dg", "dz"):
         assert np.array_equal(a[k], b[k]), k
         assert np.array_equal(a[k], c[k]), k
         assert np.array_equal(a[k], e[k]), k
+        assert np.array_equal(a[k], f[k]), k
 
 
 def test_tuned_plan_gives_identical_results():
@@ -212,7 +229,7 @@ def test_tuned_plan_gives_identical_results():
     layer.forward(wr, wg, wu, wd, x, y0, ws, True)
     assert layer.tile_plan() == -1
     plan = layer.tune_forward(wr, wg, wu, wd, x, y1, ws, True)
-    assert plan >= 0 and (plan & ~0x3F3F) == 0 and layer.tile_plan() == plan
+    assert plan >= 0 and (plan & ~63) == 0 and layer.tile_plan() == plan
     assert torch.equal(y0, y1)
     dx = torch.empty_like(x); dwr = torch.empty(wr.shape, dtype=torch.float32, device=dev)
     dwg, dwu, dwd = (torch.empty_like(w) for w in (wg, wu, wd))

@@ -1,8 +1,9 @@
 """modse_route_static_scratch: routing for callers that may not allocate device memory
 (plugins inside a framework callback, code inside a pool it does not own).  Its scratch is a
 fixed array in the library, so this checks - through the C ABI, twice in a row on different
-batches - that it returns exactly what the workspace-based modse_forward returns, and that a
-batch too large for the array is refused instead of overrunning it.
+batches - that it returns exactly what the workspace-based modse_forward returns and what the
+fp64 oracle's router returns, and that a batch too large for the array is refused instead of
+overrunning it.
 
 Collected last on purpose: a failure here leaves every other test already run."""
 import ctypes
@@ -10,7 +11,10 @@ import ctypes
 import numpy as np
 import pytest
 
+from oracle import modse_oracle as O
 from paper_2409_12210_b200 import inputs as I
+
+import helpers as H
 
 pytestmark = pytest.mark.gpu
 
@@ -43,13 +47,17 @@ def test_two_calls_in_a_row_match_the_workspace_path(name):
         base = I.LayerConfig("na_bf16", "bf16", 256, (128, 384, 192, 320), 2, 1000, seed=5, weight_std=0.05)
         cfgs = [base, I.LayerConfig("na_bf16_b", "bf16", 256, (128, 384, 192, 320), 2, 333, seed=6, weight_std=0.05)]
     for cfg in cfgs:                                   # second call reuses the array the first one left dirty
-        inp = I.generate(cfg)
+        inp, _ = H.screened(cfg)                        # near-tie tokens re-drawn, as in every parity test
         ref, x, wr = routing_via_forward(inp)
         got = B.route_static_scratch(x, wr, cfg.top_k)
         torch.cuda.synchronize()
         for key in ("topk_idx", "counts", "counts_slot", "offsets", "row_of", "token_of"):
             np.testing.assert_array_equal(got[key].cpu().numpy(), ref[key], err_msg=f"{cfg.name}:{key}")
         np.testing.assert_array_equal(got["topk_gate"].cpu().numpy(), ref["topk_gate"])   # same kernels: same bits
+        assert B.route_static_scratch_status() == B.MODSE_OK
+        # and against the oracle's router (Eq. 2-3): tables bit-exact, gates within the derived bound
+        rt = O.route(np.asarray(inp.x, np.float64), np.asarray(inp.w_router, np.float64), cfg.top_k)
+        H.check_routing({k: v.cpu().numpy() for k, v in got.items()}, rt, inp)
 
 
 def test_batches_beyond_the_fixed_array_are_refused():
