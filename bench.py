@@ -325,9 +325,12 @@ def main():
                 self.extra.append((rn(tuple(self.wr.shape), wstd), rn(tuple(self.wg.shape), wstd),
                                    rn(tuple(self.wu.shape), wstd), rn(tuple(self.wd.shape), wstd),
                                    rn(tuple(self.x.shape), 1.0), rn(tuple(self.x.shape), 1.0)))
-            self.y, self.dx = torch.empty_like(self.x), torch.empty_like(self.x)
+            odt = torch.float32 if args.out_f32 else dt
+            self.y, self.dx = torch.empty(self.x.shape, dtype=odt, device=dev), torch.empty(self.x.shape, dtype=odt, device=dev)
             self.dwr = torch.empty(self.wr.shape, dtype=torch.float32, device=dev)
-            self.dwg, self.dwu, self.dwd = (torch.empty_like(w) for w in (self.wg, self.wu, self.wd))
+            self.dwg, self.dwu, self.dwd = (torch.empty(w.shape, dtype=odt, device=dev) for w in (self.wg, self.wu, self.wd))
+            self.layer.set_output_f32(args.out_f32)
+            self.layer.set_fusion(args.fuse)
             self.bwd = c.backward
             if args.noise_gate:
                 w_noise = rn(tuple(self.wr.shape), c.d_model ** -0.5)
@@ -480,7 +483,7 @@ def main():
     # ---- end to end: pinned host inputs in, results out, every step ----
     dy = main_rep.dy
     hx, hdy = torch.from_numpy(inp.x).to(dt).pin_memory(), torch.from_numpy(inp.dy).to(dt).pin_memory()
-    hy, hdx = torch.empty_like(hx).pin_memory(), torch.empty_like(hx).pin_memory()
+    hy, hdx = torch.empty_like(main_rep.y, device="cpu").pin_memory(), torch.empty_like(main_rep.y, device="cpu").pin_memory()
     h2d = hx.numel() * hx.element_size() * (2 if do_bwd else 1)
     d2h = hy.numel() * hy.element_size() * (2 if do_bwd else 1)
 
@@ -489,7 +492,7 @@ def main():
     # that prefetches the next batch would.
     s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
     xin, dyin = [torch.empty_like(x) for _ in range(2)], [torch.empty_like(x) for _ in range(2)]
-    yout, dxout = [torch.empty_like(x) for _ in range(2)], [torch.empty_like(x) for _ in range(2)]
+    yout, dxout = [torch.empty_like(main_rep.y) for _ in range(2)], [torch.empty_like(main_rep.y) for _ in range(2)]
     E = lambda: [torch.cuda.Event() for _ in range(2)]
     ev_in, ev_done, ev_out = E(), E(), E()
 
@@ -594,7 +597,8 @@ def main():
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "d_model": d, "ffn_sizes": list(cfg.ffn_sizes), "top_k": cfg.top_k,
                    "n_tokens": T, "layers": L, "noise_gate": bool(args.noise_gate), "aux_alpha": args.aux_alpha,
-                   "tile_plan": tile_plan,
+                   "tile_plan": tile_plan, "dynamic_tiles": not args.static_tiles, "fuse": args.fuse,
+                   "outputs": "fp32" if args.out_f32 else cfg.dtype,
                    "e2e_copies": "x, dY in and y, dx out of layer 0" if L > 1 else "x, dY in; y, dx out", "pass": "fwd+bwd" if do_bwd else "fwd", "parallelism": f"replicas x{world}",
                    "l2": f"inputs larger than L2: {weight_mb * L:.0f} MB of expert weights and {act_mb * L:.0f} MB of "
                          f"permuted activations are streamed per step (L2: 126 MB)"},

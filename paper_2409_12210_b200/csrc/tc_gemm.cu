@@ -33,11 +33,15 @@
 // sp = B * silu'(A) and sq = silu(A) (bf16): then dA = dHm * sp, dB = dHm * sq, one
 // rounded factor each instead of two rounded pre-activations.
 //
-// Activations that have the hidden axis as their width (Hm, sp, sq, dA, dB)
-// are stored as panels: for expert e, panel pc holds columns [64 pc, 64 pc + 64)
-// of all cp rows contiguously, so that a single two-dimensional tensor map with
-// 128-byte rows describes the whole buffer although the row length h differs
-// from expert to expert.
+// Activations that have the hidden axis as their width and feed an MMA (Hm, dA,
+// dB) are stored as panels: for expert e, panel pc holds columns [64 pc,
+// 64 pc + 64) of all cp rows contiguously, so that a single two-dimensional
+// tensor map with 128-byte rows describes the whole buffer although the row
+// length h differs from expert to expert.  sp and sq travel only from one
+// epilogue to another, so they are stored the way an epilogue warp holds them:
+// in blocks of 32 rows x 32 columns (2 KB), inside a block the 16-byte piece q
+// of row r at byte q * 512 + r * 16.  A warp then writes and reads a block with
+// four fully coalesced 512-byte accesses and no transposition.
 //
 // Tile order: experts by decreasing K, so the long tiles of wide experts (or of
 // experts with many tokens) start first and the short ones fill the tail - the
@@ -579,8 +583,6 @@ __device__ __forceinline__ void untranspose_rows(unsigned char *stg, int lane, c
     __syncwarp();
 }
 
-// Called before the accumulator of a tile is ready: asks L2 for what the epilogue will read from
-// global memory (only the down dgrad reads: the saved SwiGLU factors of its row, and Hm for the row dot).
 // The tile's 32-column chunks are split into NQ contiguous runs, one per warp of the lane quadrant.
 template <int NQ>
 __device__ __forceinline__ void chunk_range(int ncols, int cq, int &c_begin, int &c_end)
@@ -588,22 +590,6 @@ __device__ __forceinline__ void chunk_range(int ncols, int cq, int &c_begin, int
     const int per = ((ncols >> 5) + NQ - 1) / NQ;
     c_begin = min(ncols, cq * per * 32);
     c_end = min(ncols, c_begin + per * 32);
-}
-
-template <int KIND, int VAR, int NQ>
-__device__ __forceinline__ void epilogue_prefetch(const TcParams &prm, const Tile &t, int row, int cq)
-{
-    if constexpr (KIND == TcDownDgrad) {
-        int c_begin, c_end;
-        chunk_range<NQ>(t.ncols, cq, c_begin, c_end);
-        for (int c = c_begin; c < c_end; c += 32) {
-            const int col = t.n0 + c;
-            const size_t idx = ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.sp + idx));
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.sq + idx));
-            if constexpr (VAR == 1) asm volatile("prefetch.global.L2 [%0];" ::"l"(prm.hm + idx));
-        }
-    }
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
@@ -626,6 +612,10 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
         const int col = t.n0 + c;
         return ((size_t)(t.pbase + (col >> 6) * t.cp + t.m0 + row) << 6) + (col & 63);
     };
+    // first element of the 32 x 32 block of sp / sq that holds this warp's rows and columns t.n0 + c ..
+    auto block_index = [&](int c) {
+        return ((size_t)t.pbase << 6) + ((size_t)((t.n0 + c) >> 5) * (size_t)(t.cp >> 5) + (size_t)((t.m0 + row) >> 5)) * 1024;
+    };
     if constexpr (KIND == TcUpGate) {
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
         for (int c = c_first; c < c_end; c += c_step) {
@@ -645,8 +635,13 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
                     sp[i] = bv * sg * (1.0f + av * (1.0f - sg));
                     hm[i] = gate * (sq[i] * bv);
                 }
-                store_bf16x32_staged(stg, lane, prm.sp + idx, 64, sp);
-                store_bf16x32_staged(stg, lane, prm.sq + idx, 64, sq);
+                uint4 wp[4], wq[4];
+                pack_bf16x32(sp, wp);
+                pack_bf16x32(sq, wq);
+                const size_t blk = block_index(c);
+                uint4 *dp = reinterpret_cast<uint4 *>(prm.sp + blk) + lane, *dq = reinterpret_cast<uint4 *>(prm.sq + blk) + lane;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { dp[q * 32] = wp[q]; dq[q * 32] = wq[q]; }
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
@@ -689,12 +684,17 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
         // chunk are fetched while this one is computed
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
         float rowdot = 0.f;                // VAR 1: sum over this thread's columns of acc * Hm
-        uint4 praw[4], qraw[4], hraw[4];   // transposed: entry j belongs to row 8j + lane/4 of this warp
+        uint4 pown[4], qown[4];            // this thread's row of the saved factors (block layout: no transposition)
+        uint4 hraw[4];                     // Hm, transposed: entry j belongs to row 8j + lane/4 of this warp
+        auto load_block = [&](const __nv_bfloat16 *base, int c, uint4 (&v)[4]) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(base + block_index(c)) + lane;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = src[q * 32];
+        };
         if (c_first < c_end) {
-            const size_t idx = panel_index(c_first);
-            load_bf16x32_transposed(prm.sp + idx, 64, lane, praw);
-            load_bf16x32_transposed(prm.sq + idx, 64, lane, qraw);
-            if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + idx, 64, lane, hraw);
+            load_block(prm.sp, c_first, pown);
+            load_block(prm.sq, c_first, qown);
+            if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + panel_index(c_first), 64, lane, hraw);
         }
         for (int c = c_first; c < c_end; c += c_step) {
             uint32_t r[32];
@@ -702,14 +702,10 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             uint4 pn[4], qn[4], hn[4];
             const bool more = c + c_step < c_end;
             if (more) {
-                const size_t nidx = panel_index(c + c_step);
-                load_bf16x32_transposed(prm.sp + nidx, 64, lane, pn);
-                load_bf16x32_transposed(prm.sq + nidx, 64, lane, qn);
-                if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + nidx, 64, lane, hn);
+                load_block(prm.sp, c + c_step, pn);
+                load_block(prm.sq, c + c_step, qn);
+                if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + panel_index(c + c_step), 64, lane, hn);
             }
-            uint4 pown[4], qown[4];
-            untranspose_rows(stg, lane, praw, pown);
-            untranspose_rows(stg, lane, qraw, qown);
             tmem_ld_wait();
             if constexpr (VAR == 1) {
                 uint4 hown[4];
@@ -745,7 +741,7 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             store_bf16x32_staged(stg, lane, prm.db + idx, 64, db);
             if (more) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) { praw[i] = pn[i]; qraw[i] = qn[i]; }
+                for (int i = 0; i < 4; ++i) { pown[i] = pn[i]; qown[i] = qn[i]; }
                 if constexpr (VAR == 1) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) hraw[i] = hn[i];
@@ -1095,7 +1091,6 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
             if constexpr (!WIDE) {
                 const int acc = it & 1;
                 const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
-                epilogue_prefetch<KIND, VAR, NQ>(prm, t, row, cq);
                 if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, wc)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
@@ -1103,7 +1098,6 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
                 tc_fence_before();
                 mbar_arrive(smem_u32(&st->tmem_empty[acc]));
             } else {
-                epilogue_prefetch<KIND, VAR, NQ>(prm, t, row, cq);
                 if (!mbar_wait(smem_u32(&st->tmem_full[0]), (uint32_t)it & 1u, wc)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16);
@@ -1112,7 +1106,6 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
                 mbar_arrive(smem_u32(&st->tmem_empty[0]));
                 if (t.a_boxes_peer > 0) {
                     const Tile t1 = second_half(t);
-                    epilogue_prefetch<KIND, VAR, NQ>(prm, t1, row, cq);
                     epilogue_row<KIND, VAR, NQ>(prm, t1, tacc + kAccCols, row, lane, cq, stg);
                     tc_fence_before();
                     mbar_arrive(smem_u32(&st->tmem_empty[1]));
