@@ -86,7 +86,7 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
         L.dz = take(kT * 4);
         L.du = take((size_t)T * N * 4);
         L.dgamma_partial = take((size_t)L.nblk_bwd * 4);
-        L.dwr_partial = take((size_t)L.nblk_bwd * N * m.d * 4);
+        L.dwr_partial = take((size_t)((T + kDwrTokB - 1) / kDwrTokB) * N * m.d * 4);
         L.dyp = take((size_t)L.Pmax * m.d * esz);
         L.da = take(L.hb * esz);
         L.db = take(L.hb * esz);

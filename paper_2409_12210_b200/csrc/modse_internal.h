@@ -15,6 +15,7 @@ constexpr int kMaxExperts = 256;
 constexpr int kRowPad = 128;        // every expert group is padded to a multiple of this many rows
 constexpr int kRouterTokB = 64;     // tokens per block in the router / rank kernels
 constexpr int kRouterBwdTokB = 128; // tokens per block in the router backward kernel
+constexpr int kDwrTokB = 64;        // tokens per partial sum of dW_router = dz^T x
 constexpr int kPanel = 64;          // hidden-axis panel width of the bf16 activation layout
 
 // Device status word values (first int of the workspace).  Ints 4..9 of the same 64-byte block are the

@@ -13,8 +13,8 @@
 //                      that the sum is rounded to the layer type only once.)
 //   dg_permute_kernel  dg[t,j] = <dY_t, E_(t,j)>, rows of dY in group order.
 //   router_dx_kernel   softmax Jacobian on the kept logits and dx assembly.
-//   router_dwr_kernel  per-block partial sums of dW_router = dz^T x, reduced in
-//                      block order by reduce_dwr_kernel (reproducible).
+//   router_dwr_kernel  per-block partial sums of dW_router = dz^T x, reduced in a
+//                      fixed order by reduce_dwr_kernel (reproducible).
 //
 // No kernel uses a floating-point atomic; every sum has a fixed order.
 #include "modse_internal.h"
@@ -896,9 +896,9 @@ router_dx_kernel(const T *__restrict__ w_router, const float *__restrict__ dxp, 
 
 // ---------------------------------------------------------------------------
 // Router backward, part 2: dW_router = dz^T x as per-block partial sums.  Block
-// (bx, by) owns tokens [128 bx, +128) and columns [256 by, +256); each thread
-// owns one column and adds its tokens in ascending order, eight experts at a
-// time, against the dense [128][8] slice of dz held in shared memory.  With `dense`
+// (bx, by) owns tokens [64 bx, +64) and 256 x (16 bytes of) columns; each thread
+// owns the columns of one 16-byte load and adds its tokens in ascending order, eight
+// experts at a time, against the dense [64][8] slice of dz held in shared memory.  With `dense`
 // set, the slice is read from that [T,N] array instead (dW_n = du^T x).
 // ---------------------------------------------------------------------------
 template <typename T>
@@ -907,19 +907,19 @@ router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const 
                   const float *__restrict__ dz, float *__restrict__ dwr_partial, const float *__restrict__ logits,
                   const int *__restrict__ counts_slot, float aux_scale, const float *__restrict__ dense)
 {
-    constexpr int CPT = (sizeof(T) == 2) ? 2 : 1;        // columns per thread: one 4-byte load either way
-    __shared__ float dzs[kRouterBwdTokB][8];
-    __shared__ int idxs[kRouterBwdTokB][2];
-    __shared__ float dzk[kRouterBwdTokB][2];
-    __shared__ float smax[kRouterBwdTokB], sinv[kRouterBwdTokB], sfp[kRouterBwdTokB];
+    constexpr int CPT = 16 / sizeof(T);                  // columns per thread: one 16-byte load
+    __shared__ __align__(16) float dzs[kDwrTokB][8];
+    __shared__ int idxs[kDwrTokB][2];
+    __shared__ float dzk[kDwrTokB][2];
+    __shared__ float smax[kDwrTokB], sinv[kDwrTokB], sfp[kDwrTokB];
     const int tid = threadIdx.x;
-    const int t0 = blockIdx.x * kRouterBwdTokB;
+    const int t0 = blockIdx.x * kDwrTokB;
     const int c = (blockIdx.y * 256 + tid) * CPT;
-    const int ntok = min(kRouterBwdTokB, Ttok - t0);
+    const int ntok = min(kDwrTokB, Ttok - t0);
     const float inv_T = 1.0f / (float)Ttok;
     if (aux_scale != 0.f && tid < ntok)
         token_softmax_stats(logits + (size_t)(t0 + tid) * N, counts_slot, N, inv_T, smax[tid], sinv[tid], sfp[tid]);
-    for (int i = tid; i < kRouterBwdTokB * 2; i += 256) {
+    for (int i = tid; i < kDwrTokB * 2; i += 256) {
         const int tl = i >> 1, j = i & 1;
         const bool ok = tl < ntok && j < k;
         idxs[tl][j] = ok ? topk_idx[(size_t)(t0 + tl) * k + j] : -1;
@@ -927,7 +927,7 @@ router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const 
     }
     for (int g0 = 0; g0 < N; g0 += 8) {
         __syncthreads();
-        for (int i = tid; i < kRouterBwdTokB * 8; i += 256) {
+        for (int i = tid; i < kDwrTokB * 8; i += 256) {
             const int tl = i >> 3, e = g0 + (i & 7);
             float v = 0.f;
             if (dense != nullptr) {
@@ -943,46 +943,61 @@ router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const 
             dzs[tl][i & 7] = v;
         }
         __syncthreads();
-        if (c < d) {
+        if (c < d) {                                   // d is a multiple of 8: a thread's columns are all inside or all outside
             float acc[8][CPT];
 #pragma unroll
             for (int i = 0; i < 8; ++i)
 #pragma unroll
                 for (int u = 0; u < CPT; ++u) acc[i][u] = 0.f;
+            const T *xc = x + (size_t)t0 * d + c;
 #pragma unroll 8
             for (int tl = 0; tl < ntok; ++tl) {
-                float xv[CPT];
+                float xv[8];
                 if constexpr (sizeof(T) == 4) {
-                    xv[0] = reinterpret_cast<const float *>(x)[(size_t)(t0 + tl) * d + c];
+                    const float4 q = *reinterpret_cast<const float4 *>(xc + (size_t)tl * d);
+                    xv[0] = q.x; xv[1] = q.y; xv[2] = q.z; xv[3] = q.w;
                 } else {
-                    const uint32_t w = *reinterpret_cast<const uint32_t *>(
-                        reinterpret_cast<const __nv_bfloat16 *>(x) + (size_t)(t0 + tl) * d + c);
-                    xv[0] = __uint_as_float(w << 16);
-                    xv[CPT - 1] = __uint_as_float(w & 0xFFFF0000u);
+                    load8(xc + (size_t)tl * d, xv);
                 }
+                const float4 za = *reinterpret_cast<const float4 *>(&dzs[tl][0]);
+                const float4 zb = *reinterpret_cast<const float4 *>(&dzs[tl][4]);
+                const float zz[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
 #pragma unroll
-                    for (int u = 0; u < CPT; ++u) acc[i][u] = fmaf(dzs[tl][i], xv[u], acc[i][u]);
+                    for (int u = 0; u < CPT; ++u) acc[i][u] = fmaf(zz[i], xv[u], acc[i][u]);
             }
 #pragma unroll
             for (int i = 0; i < 8; ++i)
-                if (g0 + i < N)
+                if (g0 + i < N) {
+                    float *dst = dwr_partial + ((size_t)blockIdx.x * N + g0 + i) * d + c;
 #pragma unroll
-                    for (int u = 0; u < CPT; ++u)
-                        dwr_partial[((size_t)blockIdx.x * N + g0 + i) * d + c + u] = acc[i][u];
+                    for (int u = 0; u < CPT; u += 4)
+                        *reinterpret_cast<float4 *>(dst + u) = make_float4(acc[i][u], acc[i][u + 1], acc[i][u + 2], acc[i][u + 3]);
+                }
         }
     }
 }
 
+// Sums the per-block partials in a fixed order: warp p of a block adds the partials b = p, p + 8, ... of 32
+// elements, then the eight warp sums are added in warp order.
 __global__ void __launch_bounds__(256)
 reduce_dwr_kernel(const float *__restrict__ partial, int nblk, int n, float *__restrict__ dwr)
 {
-    const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i >= n) return;
+    __shared__ float part[8][32];
+    const int lane = threadIdx.x & 31, p = threadIdx.x >> 5;
+    const int i = blockIdx.x * 32 + lane;
     float s = 0.f;
-    for (int b = 0; b < nblk; ++b) s += partial[(size_t)b * n + i];
-    dwr[i] = s;
+    if (i < n)
+        for (int b = p; b < nblk; b += 8) s += partial[(size_t)b * n + i];
+    part[p][lane] = s;
+    __syncthreads();
+    if (p == 0 && i < n) {
+        float acc = part[0][lane];
+#pragma unroll
+        for (int q = 1; q < 8; ++q) acc += part[q][lane];
+        dwr[i] = acc;
+    }
 }
 
 }  // namespace
@@ -1168,7 +1183,8 @@ cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *
             (__nv_bfloat16 *)dx, m.N, p.logits, p.counts_slot, aux_scale, (const __nv_bfloat16 *)ng.w_noise, du, Pmax, hs,
             p.status);
     MODSE_LAUNCH_CHECK();
-    dim3 grid(nblk_bwd, dt == MODSE_F32 ? (m.d + 255) / 256 : (m.d + 511) / 512);
+    const int nblk_dwr = (T + kDwrTokB - 1) / kDwrTokB;
+    dim3 grid(nblk_dwr, dt == MODSE_F32 ? (m.d + 1023) / 1024 : (m.d + 2047) / 2048);
     const int n = m.N * m.d;
     // pass 0: dW_router = dz^T x;  pass 1 (second term only): dW_n = du^T x through the same partial buffer
     for (int pass = 0; pass < (noise ? 2 : 1); ++pass) {
@@ -1182,7 +1198,7 @@ cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *
                                                                   p.topk_idx, p.dz, p.dwr_partial, p.logits,
                                                                   p.counts_slot, ascale, dense);
         MODSE_LAUNCH_CHECK();
-        reduce_dwr_kernel<<<(n + 255) / 256, 256, 0, s>>>(p.dwr_partial, nblk_bwd, n, pass ? ng.dw_noise : dw_router);
+        reduce_dwr_kernel<<<(n + 31) / 32, 256, 0, s>>>(p.dwr_partial, nblk_dwr, n, pass ? ng.dw_noise : dw_router);
         MODSE_LAUNCH_CHECK();
     }
     return cudaSuccess;
