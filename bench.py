@@ -259,6 +259,8 @@ def main():
                     help="tuning: bit k set = grouped product k on 256-row tiles (skips the set-up tuning call)")
     ap.add_argument("--static-tiles", action="store_true",
                     help="tuning: deal tiles to the CTAs round-robin instead of handing them out from a counter")
+    ap.add_argument("--epi16", type=int, nargs=2, default=None, metavar=("MASK128", "MASK256"),
+                    help="tuning: bit k set = grouped product k runs sixteen epilogue warps on 128- / 256-row tiles")
     ap.add_argument("--fuse", type=int, default=0,
                     help="fusions across the permutation (sum of 1 gather, 2 dg row dot, 4 scatter-add; see modse.h)")
     ap.add_argument("--out-f32", action="store_true", help="write y, dx and the expert weight gradients as fp32")
@@ -287,6 +289,8 @@ def main():
         B.debug_set_default_tile_plan(args.tile_plan)
     if args.static_tiles:
         B.debug_set_dynamic_tiles(False)
+    if args.epi16 is not None:
+        B.debug_set_epilogue_warps(args.epi16[0], args.epi16[1])
     dev = torch.device("cuda", local_rank)
 
     inp = I.generate(cfg)
@@ -597,7 +601,7 @@ def main():
         "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "d_model": d, "ffn_sizes": list(cfg.ffn_sizes), "top_k": cfg.top_k,
                    "n_tokens": T, "layers": L, "noise_gate": bool(args.noise_gate), "aux_alpha": args.aux_alpha,
-                   "tile_plan": tile_plan, "dynamic_tiles": not args.static_tiles, "fuse": args.fuse,
+                   "tile_plan": tile_plan, "dynamic_tiles": not args.static_tiles, "epi16": args.epi16, "fuse": args.fuse,
                    "outputs": "fp32" if args.out_f32 else cfg.dtype,
                    "e2e_copies": "x, dY in and y, dx out of layer 0" if L > 1 else "x, dY in; y, dx out", "pass": "fwd+bwd" if do_bwd else "fwd", "parallelism": f"replicas x{world}",
                    "l2": f"inputs larger than L2: {weight_mb * L:.0f} MB of expert weights and {act_mb * L:.0f} MB of "

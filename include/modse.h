@@ -317,6 +317,13 @@ void modse_debug_set_default_tile_plan(int plan);
  * counter in the workspace; 0 - the tiles are dealt to the CTAs round-robin.  Same results either way.   */
 void modse_debug_set_dynamic_tiles(int on);
 
+/* Tuning aid, process-wide: how many warps of a CTA run the epilogue of a grouped product.  Bit k of mask_128
+ * (mask_256) set: product k (numbered as in modse_get_tile_plan) runs sixteen epilogue warps when it is on
+ * 128-row (256-row) tiles, clear: eight.  Default: sixteen for the up/gate product and the down dgrad on 256-row
+ * tiles (mask_256 = 5), eight elsewhere.  Same results either way, except that the gate gradient of
+ * MODSE_FUSE_DG_ROWDOT is summed from twice as many partials (same tolerance).                               */
+void modse_debug_set_epilogue_warps(int mask_128, int mask_256);
+
 /* Failure-path aids, process-wide.  Every wait inside a kernel gives up after a limit (default 2000 ms),
  * records MODSE_ERR_DEVICE_TIMEOUT in the status word, lets its copies in flight land, frees its tensor
  * memory and returns; modse_debug_set_wait_limit_ms changes the limit (1..60000).

@@ -119,6 +119,8 @@ def load():
     lib.modse_debug_set_default_tile_plan.argtypes = [ci]
     lib.modse_debug_set_dynamic_tiles.restype = None
     lib.modse_debug_set_dynamic_tiles.argtypes = [ci]
+    lib.modse_debug_set_epilogue_warps.restype = None
+    lib.modse_debug_set_epilogue_warps.argtypes = [ci, ci]
     lib.modse_debug_set_wait_limit_ms.restype = None
     lib.modse_debug_set_wait_limit_ms.argtypes = [ci]
     lib.modse_debug_skip_tile_loads.restype = None
@@ -184,6 +186,10 @@ def debug_set_default_tile_plan(plan: int) -> None:
 
 def debug_set_dynamic_tiles(on: bool) -> None:
     load().modse_debug_set_dynamic_tiles(int(bool(on)))
+
+
+def debug_set_epilogue_warps(mask_128: int, mask_256: int) -> None:
+    load().modse_debug_set_epilogue_warps(int(mask_128), int(mask_256))
 
 
 def debug_set_wait_limit_ms(ms: int) -> None:

@@ -91,7 +91,7 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
         L.da = take(L.hb * esz);
         L.db = take(L.hb * esz);
         L.dxp = take((size_t)L.Pmax * m.d * 4);   // fp32 for every layer type
-        L.dg_slots = 2 * ((h_desc[0] + 255) / 256);
+        L.dg_slots = 4 * ((h_desc[0] + 255) / 256);
         L.dg_part = take((size_t)L.dg_slots * L.Pmax * 4);
     } else if (esz == 4) {
         // the fp32 path always materialises the two pre-activations
@@ -677,6 +677,7 @@ void modse_debug_use_fma_path(int on) { tc_set_force_simt(on); }
 void modse_debug_set_default_tile_plan(int plan) { tc_set_default_plan(plan); }
 
 void modse_debug_set_dynamic_tiles(int on) { tc_set_dynamic_tiles(on); }
+void modse_debug_set_epilogue_warps(int mask_128, int mask_256) { tc_set_epilogue_warps16(mask_128, mask_256); }
 
 void modse_debug_set_wait_limit_ms(int ms) { tc_set_wait_limit_ms(ms); }
 

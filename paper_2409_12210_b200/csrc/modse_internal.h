@@ -40,7 +40,7 @@ struct WsLayout {
     size_t status, topk_idx, topk_gate, counts, counts_slot, offsets, poffsets, ebase, row_of, token_of,
         prow_of, ptoken_of, pgate, block_counts, logits, aux_partial, noise_u, du, dgamma_partial, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
         dg_part, total;
-    int dg_slots;                    // partial row dots per padded row (two per 256-column tile of the widest expert)
+    int dg_slots;                    // partial row dots per padded row (up to four per 256-column tile of the widest expert)
     int n_canary;
     size_t canary[kMaxCanaries];     // byte offsets of the guard blocks
 };

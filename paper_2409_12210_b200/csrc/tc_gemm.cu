@@ -17,11 +17,15 @@
 // next), and 256 rows (two 128-row halves that share the column operand, 2/3 of
 // the shared-memory traffic per FLOP, but both accumulators belong to one tile).
 //
-// Roles inside a CTA (352 threads): warp 0 issues TMA loads into a ring of
-// shared-memory stages (boxes of 64 elements x 64 or 128 rows, 128-byte
-// swizzle), warp 1 issues tcgen05.mma, warp 2 hands out tiles, warps 3-10 read
-// the accumulator with tcgen05.ld (two warps per TMEM lane quadrant, each half
-// of the tile's columns) and run the fused epilogue.  Operands are consumed either K-major or MN-major
+// Roles inside a CTA: warp 0 issues TMA loads into a ring of shared-memory
+// stages (boxes of 64 elements x 64 or 128 rows, 128-byte swizzle), warp 1
+// issues tcgen05.mma, warp 2 hands out tiles, warp 3 idles, and 8 or 16 epilogue
+// warps (from warp 4 on) read the accumulator with tcgen05.ld - two or four warps
+// per TMEM lane quadrant, each a run of the tile's columns - and run the fused
+// epilogue.  A 256-row tile owns both accumulators, so its epilogue is exposed:
+// there sixteen warps (four per scheduler) hide the latencies of the epilogue's
+// loads, special-function chains and stores that eight cannot.
+// Operands are consumed either K-major or MN-major
 // straight from their row-major buffers (the instruction descriptor carries the
 // major-ness), so the backward pass needs no transposed copies.
 //
@@ -68,6 +72,7 @@ static int g_default_plan = kTcDefaultPlan;
 static int g_dynamic_tiles = 1;
 static int g_wait_limit_ms = 2000;
 static int g_skip_kind = -1, g_skip_tile = -1;
+static int g_epi16_narrow = 0, g_epi16_wide = kTcDefaultEpi16Wide;   // bit per product: sixteen epilogue warps
 
 bool tc_force_simt() { return g_force_simt != 0; }
 void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
@@ -76,20 +81,26 @@ int tc_default_plan() { return g_default_plan; }
 void tc_set_dynamic_tiles(int on) { g_dynamic_tiles = on ? 1 : 0; }
 void tc_set_wait_limit_ms(int ms) { g_wait_limit_ms = ms < 1 ? 1 : (ms > 60000 ? 60000 : ms); }
 void tc_set_skip_tile(int kind, int tile) { g_skip_kind = kind; g_skip_tile = tile; }
+void tc_set_epilogue_warps16(int narrow_mask, int wide_mask)
+{
+    g_epi16_narrow = narrow_mask & kTcPlanBits;
+    g_epi16_wide = wide_mask & kTcPlanBits;
+}
+int tc_epilogue_warps(TcKind kind, bool wide) { return (((wide ? g_epi16_wide : g_epi16_narrow) >> (int)kind) & 1) ? 16 : 8; }
 
 namespace {
 
 constexpr int kBoxBytes = 64 * 64 * 2;           // one TMA box: 64 rows of 128 bytes
 constexpr int kARegion = 2 * kBoxBytes;          // 128 rows (or 128 MN elements) x 64 K
 constexpr int kBRegion = 4 * kBoxBytes;          // up to 256 rows x 64 K
-constexpr int kEpiWarps = 8;
-constexpr int kFirstEpiWarp = 3;
-constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);   // TMA warp, MMA warp, tile warp, eight epilogue warps
+constexpr int kFirstEpiWarp = 4;                 // warps 0-2: TMA, MMA, tile hand-out; warp 3 idles (the epilogue starts on a warpgroup)
+constexpr int kMaxEpiWarps = 16;
+template <int EPI> constexpr int threads_of() { return 32 * (kFirstEpiWarp + EPI); }
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 256;
 constexpr int kEpiRowBytes = 64;                 // a 32-element bf16 chunk of one row; 16-byte pieces XOR-swizzled
 constexpr int kEpiBufBytes = 32 * kEpiRowBytes;  // one warp's 32 rows: 2 KB
-constexpr int kEpiBytes = kEpiWarps * kEpiBufBytes;   // one transposing buffer per epilogue warp
+template <int EPI> constexpr int epi_bytes() { return EPI * kEpiBufBytes; }   // one transposing buffer per epilogue warp
 constexpr int kTileQ = 4;                        // tile indices in flight between the producer and the other roles
 
 // 128-row tiles: 4 stages of 16 KB rows + 32 KB columns.  256-row tiles: 3 stages of 2 x 16 KB rows + 32 KB columns.
@@ -131,11 +142,12 @@ struct SmemTail {
     int tstart[kMaxExperts + 1];
     unsigned short order[kMaxExperts];
 };
-template <bool WIDE> constexpr size_t smem_bytes()
+template <bool WIDE, int EPI> constexpr size_t smem_bytes()
 {
-    return 1024 + (size_t)Shape<WIDE>::kStages * Shape<WIDE>::kStageBytes + kEpiBytes + sizeof(SmemTail);
+    return 1024 + (size_t)Shape<WIDE>::kStages * Shape<WIDE>::kStageBytes + epi_bytes<EPI>() + sizeof(SmemTail);
 }
-static_assert(smem_bytes<false>() <= 232448 && smem_bytes<true>() <= 232448, "shared memory per CTA");
+static_assert(smem_bytes<false, kMaxEpiWarps>() <= 232448 && smem_bytes<true, kMaxEpiWarps>() <= 232448,
+              "shared memory per CTA");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -248,6 +260,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }
@@ -479,6 +501,12 @@ __device__ __forceinline__ void pack_bf16x32(const float (&v)[32], uint4 (&w4)[4
     }
 }
 
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&t);
+}
+
 // Row-by-row stores of a warp's chunk would touch 32 lines with 16 bytes each per instruction, so the chunk is
 // transposed through shared memory: afterwards four neighbouring lanes cover the 64 bytes of one row and an
 // instruction moves eight whole 64-byte row segments.  `own` points at this thread's own row chunk.
@@ -617,39 +645,61 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
         return ((size_t)t.pbase << 6) + ((size_t)((t.n0 + c) >> 5) * (size_t)(t.cp >> 5) + (size_t)((t.m0 + row) >> 5)) * 1024;
     };
     if constexpr (KIND == TcUpGate) {
+        // 32-column chunks in two halves of 16 accumulator columns (registers: sixteen epilogue warps leave 96
+        // per thread); the chunk's gated hidden values are kept packed and leave as 64-byte row segments
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
         for (int c = c_first; c < c_end; c += c_step) {
-            uint32_t ra[32], rb[32];
-            tmem_ld32(tacc + c, ra);
-            tmem_ld32(tacc + t.ncols + c, rb);
-            tmem_ld_wait();
-            const size_t idx = panel_index(c);
-            float hm[32];
+            uint4 hw4[4];
+            uint4 *dp = nullptr, *dq = nullptr;
             if (prm.save) {
-                float sp[32], sq[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float av = __uint_as_float(ra[i]), bv = __uint_as_float(rb[i]);
-                    const float sg = __fdividef(1.0f, 1.0f + __expf(-av));   // ex2 + rcp: a full-precision division here slows the MMA warp
-                    sq[i] = av * sg;
-                    sp[i] = bv * sg * (1.0f + av * (1.0f - sg));
-                    hm[i] = gate * (sq[i] * bv);
-                }
-                uint4 wp[4], wq[4];
-                pack_bf16x32(sp, wp);
-                pack_bf16x32(sq, wq);
                 const size_t blk = block_index(c);
-                uint4 *dp = reinterpret_cast<uint4 *>(prm.sp + blk) + lane, *dq = reinterpret_cast<uint4 *>(prm.sq + blk) + lane;
-#pragma unroll
-                for (int q = 0; q < 4; ++q) { dp[q * 32] = wp[q]; dq[q * 32] = wq[q]; }
-            } else {
-#pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const float av = __uint_as_float(ra[i]), bv = __uint_as_float(rb[i]);
-                    hm[i] = gate * (av * __fdividef(1.0f, 1.0f + __expf(-av)) * bv);
-                }
+                dp = reinterpret_cast<uint4 *>(prm.sp + blk) + lane;
+                dq = reinterpret_cast<uint4 *>(prm.sq + blk) + lane;
             }
-            store_bf16x32_staged(stg, lane, prm.hm + idx, 64, hm);
+#pragma unroll
+            for (int s2 = 0; s2 < 2; ++s2) {
+                uint32_t ra[16], rb[16];
+                tmem_ld16(tacc + c + 16 * s2, ra);
+                tmem_ld16(tacc + t.ncols + c + 16 * s2, rb);
+                tmem_ld_wait();
+                uint32_t wh[8];
+                if (prm.save) {
+                    uint32_t wp[8], wq[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float sq2[2], sp2[2], hm2[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const float av = __uint_as_float(ra[2 * i + u]), bv = __uint_as_float(rb[2 * i + u]);
+                            const float sg = __fdividef(1.0f, 1.0f + __expf(-av));   // ex2 + rcp: a full-precision division here slows the MMA warp
+                            sq2[u] = av * sg;
+                            sp2[u] = bv * sg * (1.0f + av * (1.0f - sg));
+                            hm2[u] = gate * (sq2[u] * bv);
+                        }
+                        wp[i] = pack_bf16x2(sp2[0], sp2[1]);
+                        wq[i] = pack_bf16x2(sq2[0], sq2[1]);
+                        wh[i] = pack_bf16x2(hm2[0], hm2[1]);
+                    }
+                    dp[(2 * s2) * 32] = make_uint4(wp[0], wp[1], wp[2], wp[3]);
+                    dp[(2 * s2 + 1) * 32] = make_uint4(wp[4], wp[5], wp[6], wp[7]);
+                    dq[(2 * s2) * 32] = make_uint4(wq[0], wq[1], wq[2], wq[3]);
+                    dq[(2 * s2 + 1) * 32] = make_uint4(wq[4], wq[5], wq[6], wq[7]);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        float hm2[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const float av = __uint_as_float(ra[2 * i + u]), bv = __uint_as_float(rb[2 * i + u]);
+                            hm2[u] = gate * (av * __fdividef(1.0f, 1.0f + __expf(-av)) * bv);
+                        }
+                        wh[i] = pack_bf16x2(hm2[0], hm2[1]);
+                    }
+                }
+                hw4[2 * s2] = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+                hw4[2 * s2 + 1] = make_uint4(wh[4], wh[5], wh[6], wh[7]);
+            }
+            store_u4x4_staged(stg, lane, reinterpret_cast<unsigned char *>(prm.hm + panel_index(c)), 128, hw4, 32);
         }
     } else if constexpr (KIND == TcDown || KIND == TcUpGateDgrad) {
         if constexpr (VAR == 1) {
@@ -680,77 +730,61 @@ __device__ __forceinline__ void epilogue_row(const TcParams &prm, const Tile &t,
             }
         }
     } else if constexpr (KIND == TcDownDgrad) {
-        // dA = dHm * sp, dB = dHm * sq with dHm = gate * acc; the saved factors of the next
-        // chunk are fetched while this one is computed
+        // dA = dHm * sp, dB = dHm * sq with dHm = gate * acc, 32-column chunks in two halves of 16 columns;
+        // the saved factors (and, for the row dot, Hm) of a chunk are requested before its accumulator
         const float gate = prm.pgate[t.prow0 + t.m0 + row];
         float rowdot = 0.f;                // VAR 1: sum over this thread's columns of acc * Hm
-        uint4 pown[4], qown[4];            // this thread's row of the saved factors (block layout: no transposition)
-        uint4 hraw[4];                     // Hm, transposed: entry j belongs to row 8j + lane/4 of this warp
-        auto load_block = [&](const __nv_bfloat16 *base, int c, uint4 (&v)[4]) {
-            const uint4 *src = reinterpret_cast<const uint4 *>(base + block_index(c)) + lane;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) v[q] = src[q * 32];
-        };
-        if (c_first < c_end) {
-            load_block(prm.sp, c_first, pown);
-            load_block(prm.sq, c_first, qown);
-            if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + panel_index(c_first), 64, lane, hraw);
-        }
         for (int c = c_first; c < c_end; c += c_step) {
-            uint32_t r[32];
-            tmem_ld32(tacc + c, r);
-            uint4 pn[4], qn[4], hn[4];
-            const bool more = c + c_step < c_end;
-            if (more) {
-                load_block(prm.sp, c + c_step, pn);
-                load_block(prm.sq, c + c_step, qn);
-                if constexpr (VAR == 1) load_bf16x32_transposed(prm.hm + panel_index(c + c_step), 64, lane, hn);
-            }
-            tmem_ld_wait();
-            if constexpr (VAR == 1) {
-                uint4 hown[4];
-                untranspose_rows(stg, lane, hraw, hown);
+            const uint4 *psrc = reinterpret_cast<const uint4 *>(prm.sp + block_index(c)) + lane;
+            const uint4 *qsrc = reinterpret_cast<const uint4 *>(prm.sq + block_index(c)) + lane;
+            uint4 pown[4], qown[4];        // this thread's row of the saved factors (block layout: no transposition)
 #pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    const uint32_t hw[4] = {hown[q4].x, hown[q4].y, hown[q4].z, hown[q4].w};
+            for (int q = 0; q < 4; ++q) { pown[q] = psrc[q * 32]; qown[q] = qsrc[q * 32]; }
+            uint4 hown[4];
+            if constexpr (VAR == 1) {
+                uint4 hraw[4];             // Hm, transposed: entry j belongs to row 8j + lane/4 of this warp
+                load_bf16x32_transposed(prm.hm + panel_index(c), 64, lane, hraw);
+                untranspose_rows(stg, lane, hraw, hown);
+            }
+            uint4 da4[4], db4[4];
+#pragma unroll
+            for (int s2 = 0; s2 < 2; ++s2) {
+                uint32_t r[16];
+                tmem_ld16(tacc + c + 16 * s2, r);
+                tmem_ld_wait();
+                uint32_t wa[8], wb[8];
+#pragma unroll
+                for (int q4 = 0; q4 < 2; ++q4) {
+                    const uint4 p4 = pown[2 * s2 + q4], q4v = qown[2 * s2 + q4];
+                    const uint32_t pw[4] = {p4.x, p4.y, p4.z, p4.w};
+                    const uint32_t qw[4] = {q4v.x, q4v.y, q4v.z, q4v.w};
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int e0 = q4 * 8 + 2 * i;
-                        rowdot = fmaf(__uint_as_float(r[e0]), bf16_lo(hw[i]), rowdot);
-                        rowdot = fmaf(__uint_as_float(r[e0 + 1]), bf16_hi(hw[i]), rowdot);
+                        const float a0 = __uint_as_float(r[e0]), a1 = __uint_as_float(r[e0 + 1]);
+                        if constexpr (VAR == 1) {
+                            const uint4 h4 = hown[2 * s2 + q4];
+                            const uint32_t hw[4] = {h4.x, h4.y, h4.z, h4.w};
+                            rowdot = fmaf(a0, bf16_lo(hw[i]), rowdot);
+                            rowdot = fmaf(a1, bf16_hi(hw[i]), rowdot);
+                        }
+                        const float dh0 = gate * a0, dh1 = gate * a1;
+                        wa[q4 * 4 + i] = pack_bf16x2(dh0 * bf16_lo(pw[i]), dh1 * bf16_hi(pw[i]));
+                        wb[q4 * 4 + i] = pack_bf16x2(dh0 * bf16_lo(qw[i]), dh1 * bf16_hi(qw[i]));
                     }
                 }
+                da4[2 * s2] = make_uint4(wa[0], wa[1], wa[2], wa[3]);
+                da4[2 * s2 + 1] = make_uint4(wa[4], wa[5], wa[6], wa[7]);
+                db4[2 * s2] = make_uint4(wb[0], wb[1], wb[2], wb[3]);
+                db4[2 * s2 + 1] = make_uint4(wb[4], wb[5], wb[6], wb[7]);
             }
             const size_t idx = panel_index(c);
-            float da[32], db[32];
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                const uint32_t pw[4] = {pown[q4].x, pown[q4].y, pown[q4].z, pown[q4].w};
-                const uint32_t qw[4] = {qown[q4].x, qown[q4].y, qown[q4].z, qown[q4].w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int e0 = q4 * 8 + 2 * i;
-                    const float dh0 = gate * __uint_as_float(r[e0]), dh1 = gate * __uint_as_float(r[e0 + 1]);
-                    da[e0] = dh0 * bf16_lo(pw[i]);
-                    da[e0 + 1] = dh1 * bf16_hi(pw[i]);
-                    db[e0] = dh0 * bf16_lo(qw[i]);
-                    db[e0 + 1] = dh1 * bf16_hi(qw[i]);
-                }
-            }
-            store_bf16x32_staged(stg, lane, prm.da + idx, 64, da);
-            store_bf16x32_staged(stg, lane, prm.db + idx, 64, db);
-            if (more) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) { pown[i] = pn[i]; qown[i] = qn[i]; }
-                if constexpr (VAR == 1) {
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) hraw[i] = hn[i];
-                }
-            }
+            store_u4x4_staged(stg, lane, reinterpret_cast<unsigned char *>(prm.da + idx), 128, da4, 32);
+            store_u4x4_staged(stg, lane, reinterpret_cast<unsigned char *>(prm.db + idx), 128, db4, 32);
         }
-        // one partial per (row, 256-column tile, half of the columns); a warp without a chunk writes its zero
+        // one partial per (row, 256-column tile, run of the columns); a warp without a chunk writes its zero
         if constexpr (VAR == 1)
-            prm.dg_part[(size_t)((t.n0 >> 8) * 2 + cq) * prm.Pmax + t.prow0 + t.m0 + row] = rowdot;
+            prm.dg_part[(size_t)((t.n0 >> 8) * NQ + cq) * prm.Pmax + t.prow0 + t.m0 + row] = rowdot;
     } else if constexpr (KIND == TcDownWgrad) {
         const size_t oidx = (size_t)(t.m0 + row) * S + t.ho + t.n0;
         for (int c = c_first; c < c_end; c += c_step) {
@@ -799,7 +833,7 @@ template <int KIND, bool WIDE>
 __device__ __forceinline__ void build_schedule(const TcParams &prm, SmemTail *st, int *key, int *ntile, int tid)
 {
     const int N = prm.meta.N, d = prm.meta.d;
-    for (int e = tid; e < N; e += kThreads) {
+    for (int e = tid; e < N; e += (int)blockDim.x) {
         const int cp = prm.poffsets[e + 1] - prm.poffsets[e];
         const int h = prm.meta.hoff[e + 1] - prm.meta.hoff[e];
         int mt, nt, nk;
@@ -812,7 +846,7 @@ __device__ __forceinline__ void build_schedule(const TcParams &prm, SmemTail *st
         key[e] = nk;
     }
     __syncthreads();
-    for (int e = tid; e < N; e += kThreads) {
+    for (int e = tid; e < N; e += (int)blockDim.x) {
         int rank = 0;
         const int ke = key[e];
         for (int f = 0; f < N; ++f) {
@@ -873,11 +907,11 @@ __device__ __forceinline__ void release_tile(const TcParams &prm, SmemTail *st, 
 // warp issues one four-row gather per half and k-block), DownDgrad writes row
 // dots for dg, Down / UpGateDgrad add into token rows.
 // ---------------------------------------------------------------------------
-template <int KIND, bool WIDE, int VAR>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int KIND, bool WIDE, int VAR, int EPI>
+__global__ void __launch_bounds__(threads_of<EPI>(), 1)
 tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
 {
-    constexpr int NQ = kEpiWarps / 4;            // epilogue warps per TMEM lane quadrant
+    constexpr int NQ = EPI / 4;                  // epilogue warps per TMEM lane quadrant
     using Sh = Shape<WIDE>;
     constexpr int kStages = Sh::kStages;
     constexpr int kStageBytes = Sh::kStageBytes;
@@ -888,7 +922,7 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
     unsigned char *smem = smem_raw + pad;
     const uint32_t stage_base = raw + pad;
     unsigned char *epi_bufs = smem + (size_t)kStages * kStageBytes;
-    SmemTail *st = reinterpret_cast<SmemTail *>(epi_bufs + kEpiBytes);
+    SmemTail *st = reinterpret_cast<SmemTail *>(epi_bufs + EPI * kEpiBufBytes);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -899,12 +933,12 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
         }
         mbar_init(smem_u32(&st->tmem_full[0]), 1);
         mbar_init(smem_u32(&st->tmem_full[1]), 1);
-        mbar_init(smem_u32(&st->tmem_empty[0]), 32 * kEpiWarps);
-        mbar_init(smem_u32(&st->tmem_empty[1]), 32 * kEpiWarps);
+        mbar_init(smem_u32(&st->tmem_empty[0]), 32 * EPI);
+        mbar_init(smem_u32(&st->tmem_empty[1]), 32 * EPI);
         mbar_init(smem_u32(&st->tq_taken), 1);
         for (int s = 0; s < kTileQ; ++s) {
             mbar_init(smem_u32(&st->tq_full[s]), 1);
-            mbar_init(smem_u32(&st->tq_empty[s]), 2 + kEpiWarps);   // the TMA leader, the MMA thread and one lane of each epilogue warp
+            mbar_init(smem_u32(&st->tq_empty[s]), 2 + EPI);   // the TMA leader, the MMA thread and one lane of each epilogue warp
         }
         st->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1073,10 +1107,10 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
     } else if (warp == 2) {
         // ===================== tile hand-out =====================
         if (lane == 0 && prm.dynamic) hand_out_tiles(prm, st, total_tiles, wc);
-    } else {
-        // ===================== epilogue (warps 3 .. 10) =====================
+    } else if (warp >= kFirstEpiWarp) {
+        // ===================== epilogue =====================
         const int quad = warp & 3;                 // TMEM lane quadrant this warp may read
-        const int cq = (warp - kFirstEpiWarp) >> 2;   // which of the quadrant's two warps: the first or second half of the columns
+        const int cq = (warp - kFirstEpiWarp) >> 2;   // which of the quadrant's NQ warps: which run of the tile's columns
         const int row = quad * 32 + lane;
         unsigned char *stg = epi_bufs + (warp - kFirstEpiWarp) * kEpiBufBytes;
         int cursor = 0;
@@ -1127,14 +1161,15 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
 // Sums the partial row dots of the down dgrad in slot order and divides by the gate:
 // dg[t, j] = <dY_t W_down, Hm_row> / g = <dY_t, E_(t,j)>.  One thread per assignment.
 __global__ void __launch_bounds__(256)
-dg_finish_kernel(LayerMeta m, int Ttok, int Pmax, const int *__restrict__ topk_idx, const float *__restrict__ topk_gate,
-                 const int *__restrict__ prow_of, const float *__restrict__ dg_part, float *__restrict__ dg, int *status)
+dg_finish_kernel(LayerMeta m, int Ttok, int Pmax, int per_tile, const int *__restrict__ topk_idx,
+                 const float *__restrict__ topk_gate, const int *__restrict__ prow_of, const float *__restrict__ dg_part,
+                 float *__restrict__ dg, int *status)
 {
     const int i = blockIdx.x * 256 + threadIdx.x;
     if (i >= Ttok * m.k) return;
     const int e = topk_idx[i], prow = prow_of[i];
     if (e < 0 || e >= m.N || prow < 0 || prow >= Pmax) { atomicMax(status, kDevBounds); return; }
-    const int slots = 2 * ((m.hoff[e + 1] - m.hoff[e] + 255) / 256);     // two per 256-column tile
+    const int slots = per_tile * ((m.hoff[e + 1] - m.hoff[e] + 255) / 256);     // one per epilogue warp of a lane quadrant and 256-column tile
     float acc = 0.f;
     for (int sl = 0; sl < slots; ++sl) acc += dg_part[(size_t)sl * Pmax + prow];
     const float g = topk_gate[i];
@@ -1206,11 +1241,11 @@ bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsP
 
 namespace {
 
-template <int KIND, bool WIDE, int VAR>
+template <int KIND, bool WIDE, int VAR, int EPI>
 cudaError_t launch_one(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
 {
-    auto kern = tc_grouped_gemm<KIND, WIDE, VAR>;
-    constexpr size_t smem = smem_bytes<WIDE>();
+    auto kern = tc_grouped_gemm<KIND, WIDE, VAR, EPI>;
+    constexpr size_t smem = smem_bytes<WIDE, EPI>();
     // the shared-memory attribute of a kernel is set once per process and device
     static unsigned long long attr_done = 0;      // bit per device ordinal (devices beyond 63 set it every time)
     int dev = 0;
@@ -1221,22 +1256,30 @@ cudaError_t launch_one(const TcMaps &maps, const TcParams &prm, int grid, cudaSt
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev <= 63) attr_done |= 1ull << dev;
     }
-    kern<<<grid, kThreads, smem, s>>>(maps, prm);
+    kern<<<grid, threads_of<EPI>(), smem, s>>>(maps, prm);
     e = cudaGetLastError();
     if (e == cudaSuccess && launches) ++*launches;
     return e;
 }
 
+template <int KIND, bool WIDE, int VAR>
+cudaError_t launch_epi(const TcMaps &maps, const TcParams &prm, int grid, int epi, cudaStream_t s, int *launches)
+{
+    return epi == 16 ? launch_one<KIND, WIDE, VAR, 16>(maps, prm, grid, s, launches)
+                     : launch_one<KIND, WIDE, VAR, 8>(maps, prm, grid, s, launches);
+}
+
 template <int KIND, bool HAS_VAR>
-cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, bool wide, int var, cudaStream_t s, int *launches)
+cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, bool wide, int var, int epi, cudaStream_t s,
+                        int *launches)
 {
     if constexpr (HAS_VAR) {
         if (var)
-            return wide ? launch_one<KIND, true, 1>(maps, prm, grid, s, launches)
-                        : launch_one<KIND, false, 1>(maps, prm, grid, s, launches);
+            return wide ? launch_epi<KIND, true, 1>(maps, prm, grid, epi, s, launches)
+                        : launch_epi<KIND, false, 1>(maps, prm, grid, epi, s, launches);
     }
-    return wide ? launch_one<KIND, true, 0>(maps, prm, grid, s, launches)
-                : launch_one<KIND, false, 0>(maps, prm, grid, s, launches);
+    return wide ? launch_epi<KIND, true, 0>(maps, prm, grid, epi, s, launches)
+                : launch_epi<KIND, false, 0>(maps, prm, grid, epi, s, launches);
 }
 
 int sm_count(TcPlan &plan)
@@ -1290,20 +1333,21 @@ cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const Layer
     const int grid = sm_count(plan);
     const int mask = plan.tile_mask >= 0 ? plan.tile_mask : tc_default_plan();
     const bool wide = ((mask >> (int)kind) & 1) != 0;
+    const int epi = tc_epilogue_warps(kind, wide);
     cudaError_t e = cudaErrorInvalidValue;
     switch (kind) {
-    case TcUpGate: e = launch_kind<TcUpGate, true>(maps, prm, grid, wide, fuse & kFuseGather, s, launches); break;
-    case TcDown: e = launch_kind<TcDown, true>(maps, prm, grid, wide, fuse & kFuseScatter, s, launches); break;
-    case TcDownDgrad: e = launch_kind<TcDownDgrad, true>(maps, prm, grid, wide, fuse & kFuseDgRowdot, s, launches); break;
-    case TcDownWgrad: e = launch_kind<TcDownWgrad, false>(maps, prm, grid, wide, 0, s, launches); break;
-    case TcUpGateDgrad: e = launch_kind<TcUpGateDgrad, true>(maps, prm, grid, wide, fuse & kFuseScatter, s, launches); break;
-    case TcUpGateWgrad: e = launch_kind<TcUpGateWgrad, false>(maps, prm, grid, wide, 0, s, launches); break;
+    case TcUpGate: e = launch_kind<TcUpGate, true>(maps, prm, grid, wide, fuse & kFuseGather, epi, s, launches); break;
+    case TcDown: e = launch_kind<TcDown, true>(maps, prm, grid, wide, fuse & kFuseScatter, epi, s, launches); break;
+    case TcDownDgrad: e = launch_kind<TcDownDgrad, true>(maps, prm, grid, wide, fuse & kFuseDgRowdot, epi, s, launches); break;
+    case TcDownWgrad: e = launch_kind<TcDownWgrad, false>(maps, prm, grid, wide, 0, epi, s, launches); break;
+    case TcUpGateDgrad: e = launch_kind<TcUpGateDgrad, true>(maps, prm, grid, wide, fuse & kFuseScatter, epi, s, launches); break;
+    case TcUpGateWgrad: e = launch_kind<TcUpGateWgrad, false>(maps, prm, grid, wide, 0, epi, s, launches); break;
     }
     if (e != cudaSuccess) return e;
     if (kind == TcDownDgrad && (fuse & kFuseDgRowdot)) {
         const int n = L.T * m.k;
-        dg_finish_kernel<<<(n + 255) / 256, 256, 0, s>>>(m, L.T, L.Pmax, p.topk_idx, p.topk_gate, p.prow_of, p.dg_part, p.dg,
-                                                         p.status);
+        dg_finish_kernel<<<(n + 255) / 256, 256, 0, s>>>(m, L.T, L.Pmax, epi / 4, p.topk_idx, p.topk_gate, p.prow_of,
+                                                         p.dg_part, p.dg, p.status);
         e = cudaGetLastError();
         if (e == cudaSuccess && launches) ++*launches;
     }

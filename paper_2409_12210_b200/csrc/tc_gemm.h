@@ -22,6 +22,8 @@ enum TcKind : int {
 // long K loops (down, down wgrad, up/gate dgrad, up/gate wgrad) on 256-row tiles.
 constexpr int kTcDefaultPlan = (1 << TcDown) | (1 << TcDownWgrad) | (1 << TcUpGateDgrad) | (1 << TcUpGateWgrad);
 constexpr int kTcPlanBits = 63;
+// Epilogue warps per CTA: bit k set = product k runs sixteen of them on its 256-row tiles (eight otherwise).
+constexpr int kTcDefaultEpi16Wide = (1 << TcUpGate) | (1 << TcDownDgrad);
 
 // Optional fusions across the permutation (what lies either side of the permute / un-permute steps).
 enum : int {
@@ -67,6 +69,8 @@ void tc_set_default_plan(int mask);   // tile plan used by layers that have none
 int tc_default_plan();
 void tc_set_dynamic_tiles(int on);    // 1 (default): CTAs take tiles from a shared counter; 0: tiles are dealt statically
 void tc_set_wait_limit_ms(int ms);    // limit of every bounded wait inside the kernels (default 2000)
+void tc_set_epilogue_warps16(int narrow_mask, int wide_mask);   // bit per product: sixteen epilogue warps on 128- / 256-row tiles
+int tc_epilogue_warps(TcKind kind, bool wide);
 void tc_set_skip_tile(int kind, int tile);   // the producer of the CTA that gets `tile` of product `kind` stops there (-1: off)
 
 bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,
