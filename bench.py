@@ -67,10 +67,12 @@ def same_kernel_as_captured(stage: str, tile_plan: int) -> bool:
              "upgate_dgrad": 4, "upgate_wgrad": 5}
     if tile_plan < 0 or stage not in kinds:
         return True
-    k, default = kinds[stage], 0b111010
-    return ((tile_plan >> k) & 1) == ((default >> k) & 1)
+    k, default = kinds[stage], B_DEFAULT_TILE_PLAN
+    shape = lambda plan: 2 if (plan >> (8 + k)) & 1 else (plan >> k) & 1
+    return shape(tile_plan) == shape(default)
 
 
+B_DEFAULT_TILE_PLAN = 0x3F3A       # the library's default plan (binding.DEFAULT_TILE_PLAN)
 STAGE_BOUND = ["hbm", "hbm", "hbm", "tensor", "tensor", "hbm", "hbm", "tensor", "tensor", "tensor", "tensor", "hbm"]
 
 
@@ -256,11 +258,13 @@ def main():
     ap.add_argument("--sustained-seconds", type=float, default=2.0,
                     help="length of the extra back-to-back run that gives the power-limited figure (0: skip)")
     ap.add_argument("--tile-plan", type=int, default=None,
-                    help="tuning: bit k set = grouped product k on 256-row tiles (skips the set-up tuning call)")
+                    help="tuning: bit k set = grouped product k on one-CTA 256-row tiles, bit 8 + k = on CTA-pair "
+                         "tiles (skips the set-up tuning call)")
     ap.add_argument("--static-tiles", action="store_true",
                     help="tuning: deal tiles to the CTAs round-robin instead of handing them out from a counter")
-    ap.add_argument("--epi16", type=int, nargs=2, default=None, metavar=("MASK128", "MASK256"),
-                    help="tuning: bit k set = grouped product k runs sixteen epilogue warps on 128- / 256-row tiles")
+    ap.add_argument("--epi16", type=int, nargs=3, default=None, metavar=("MASK128", "MASK256", "MASKPAIR"),
+                    help="tuning: bit k set = grouped product k runs sixteen epilogue warps on 128-row / one-CTA "
+                         "256-row / CTA-pair tiles")
     ap.add_argument("--fuse", type=int, default=0,
                     help="fusions across the permutation (sum of 1 gather, 2 dg row dot, 4 scatter-add; see modse.h)")
     ap.add_argument("--out-f32", action="store_true", help="write y, dx and the expert weight gradients as fp32")
@@ -290,7 +294,7 @@ def main():
     if args.static_tiles:
         B.debug_set_dynamic_tiles(False)
     if args.epi16 is not None:
-        B.debug_set_epilogue_warps(args.epi16[0], args.epi16[1])
+        B.debug_set_epilogue_warps(*args.epi16)
     dev = torch.device("cuda", local_rank)
 
     inp = I.generate(cfg)

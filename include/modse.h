@@ -190,16 +190,17 @@ modse_status_t modse_set_aux_loss(modse_layer_t *layer, float alpha);
 modse_status_t modse_set_output_f32(modse_layer_t *layer, int on);
 
 /* Choice of kernel shape per device (no counterpart in the paper: a property of this implementation).
- * Each grouped product of the bf16 layer exists with 128-row and with 256-row tiles; which is faster for the
- * two forward products depends on how fast the GPU at hand feeds shared memory from L2, which differs between
- * otherwise identical boards.  modse_tune_forward runs the forward pass (arguments as modse_forward) a few
+ * Each grouped product of the bf16 layer exists with 128-row tiles, with 256-row tiles computed by one CTA and
+ * with 256-row tiles computed by a pair of CTAs; which is fastest for the two forward products depends on how
+ * fast the GPU at hand feeds shared memory from L2, which differs between otherwise identical boards.  modse_tune_forward runs the forward pass (arguments as modse_forward) a few
  * times per candidate on the caller's own buffers, times it with CUDA events, and keeps the fastest plan in
  * the layer object for all later calls.  It allocates no device memory, SYNCHRONISES the stream, and leaves y
  * and the workspace as one modse_forward would.  Results do not depend on the plan (the K order of every sum
  * is the same).  fp32 layers have one kernel shape: the call returns MODSE_OK at once.
- * modse_get_tile_plan returns the plan (-1: library default; else bit k set: product k on 256-row tiles,
- * clear: on 128-row tiles; k = 0 up/gate, 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate dgrad, 5 up/gate
- * wgrad); modse_set_tile_plan installs one (e.g. a plan found earlier on the same device). */
+ * modse_get_tile_plan returns the plan: -1 for the library default, else a bit set with, for product k (0 up/gate,
+ * 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate dgrad, 5 up/gate wgrad), bit 8 + k set: 256-row tiles computed
+ * by a pair of CTAs on neighbouring SMs; otherwise bit k set: 256-row tiles computed by one CTA, clear: 128-row
+ * tiles.  modse_set_tile_plan installs one (e.g. a plan found earlier on the same device). */
 modse_status_t modse_tune_forward(modse_layer_t *layer, modse_dtype_t dtype, const modse_weights_t *weights,
                                   const void *x, int n_tokens, void *y, void *workspace, size_t workspace_bytes,
                                   int save_for_backward, void *cuda_stream);
@@ -309,20 +310,21 @@ const char *modse_stage_name(int stage);
 void modse_debug_use_fma_path(int on);
 
 /* Tuning aid, process-wide: the tile plan (see modse_get_tile_plan) of layers that have none of their own.
- * The library's default puts products 1, 3, 4 and 5 on 256-row tiles.  Every choice gives bit-identical
- * results (the order in which each output element is summed does not depend on the tile shape).        */
+ * The library's default (0x3F3A) puts every product on CTA pairs, and, where that kernel does not apply (the
+ * row-gathering up/gate product), products 1, 3, 4 and 5 on one-CTA 256-row tiles.  Every choice gives
+ * bit-identical results (the order in which each output element is summed does not depend on the tile shape). */
 void modse_debug_set_default_tile_plan(int plan);
 
 /* Tuning aid, process-wide: 1 (default) - the CTAs of a grouped product take tiles, longest K first, from a
  * counter in the workspace; 0 - the tiles are dealt to the CTAs round-robin.  Same results either way.   */
 void modse_debug_set_dynamic_tiles(int on);
 
-/* Tuning aid, process-wide: how many warps of a CTA run the epilogue of a grouped product.  Bit k of mask_128
- * (mask_256) set: product k (numbered as in modse_get_tile_plan) runs sixteen epilogue warps when it is on
- * 128-row (256-row) tiles, clear: eight.  Default: sixteen for the up/gate product and the down dgrad on 256-row
- * tiles (mask_256 = 5), eight elsewhere.  Same results either way, except that the gate gradient of
- * MODSE_FUSE_DG_ROWDOT is summed from twice as many partials (same tolerance).                               */
-void modse_debug_set_epilogue_warps(int mask_128, int mask_256);
+/* Tuning aid, process-wide: how many warps of a CTA run the epilogue of a grouped product.  Bit k of mask_128 /
+ * mask_256 / mask_pair set: product k (numbered as in modse_get_tile_plan) runs sixteen epilogue warps when it
+ * is on 128-row tiles / one-CTA 256-row tiles / CTA-pair tiles, clear: eight.  Default: sixteen for the up/gate
+ * product and the down dgrad on one-CTA 256-row tiles (mask_256 = 5), eight elsewhere.  Same results either way,
+ * except that the gate gradient of MODSE_FUSE_DG_ROWDOT is summed from twice as many partials (same tolerance). */
+void modse_debug_set_epilogue_warps(int mask_128, int mask_256, int mask_pair);
 
 /* Failure-path aids, process-wide.  Every wait inside a kernel gives up after a limit (default 2000 ms),
  * records MODSE_ERR_DEVICE_TIMEOUT in the status word, lets its copies in flight land, frees its tensor

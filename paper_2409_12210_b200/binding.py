@@ -27,7 +27,8 @@ N_STAGES = 12
 MODSE_FUSE_GATHER = 1
 MODSE_FUSE_DG_ROWDOT = 2
 MODSE_FUSE_SCATTER = 4
-DEFAULT_TILE_PLAN = 0b111010       # products 1, 3, 4, 5 on 256-row tiles
+DEFAULT_TILE_PLAN = 0x3F3A         # every product on CTA pairs; fallback: products 1, 3, 4, 5 on one-CTA 256-row tiles
+PAIR_SHIFT = 8                     # bit 8 + k of a plan: product k on 256-row tiles computed by a pair of CTAs
 
 
 class ModseError(RuntimeError):
@@ -120,7 +121,7 @@ def load():
     lib.modse_debug_set_dynamic_tiles.restype = None
     lib.modse_debug_set_dynamic_tiles.argtypes = [ci]
     lib.modse_debug_set_epilogue_warps.restype = None
-    lib.modse_debug_set_epilogue_warps.argtypes = [ci, ci]
+    lib.modse_debug_set_epilogue_warps.argtypes = [ci, ci, ci]
     lib.modse_debug_set_wait_limit_ms.restype = None
     lib.modse_debug_set_wait_limit_ms.argtypes = [ci]
     lib.modse_debug_skip_tile_loads.restype = None
@@ -188,8 +189,8 @@ def debug_set_dynamic_tiles(on: bool) -> None:
     load().modse_debug_set_dynamic_tiles(int(bool(on)))
 
 
-def debug_set_epilogue_warps(mask_128: int, mask_256: int) -> None:
-    load().modse_debug_set_epilogue_warps(int(mask_128), int(mask_256))
+def debug_set_epilogue_warps(mask_128: int = 0, mask_256: int = 5, mask_pair: int = 0) -> None:
+    load().modse_debug_set_epilogue_warps(int(mask_128), int(mask_256), int(mask_pair))
 
 
 def debug_set_wait_limit_ms(ms: int) -> None:

@@ -610,27 +610,29 @@ modse_status_t modse_tune_forward(modse_layer_t *layer, modse_dtype_t dtype, con
     if (cudaEventCreate(&ev[1]) != cudaSuccess) { cudaEventDestroy(ev[0]); return MODSE_ERR_CUDA; }
     const int prev = layer->tc.tile_mask;
     const int base = prev >= 0 ? prev : tc_default_plan();
-    const int fwd_bits = (1 << TcUpGate) | (1 << TcDown);
-    // candidates: each forward product on 128-row or on 256-row tiles.  They are timed in
-    // interleaved rounds after a warm-up, so that the drift of the clocks under the power limit (a burst
-    // after idle, lower clocks later) does not favour whichever candidate runs first.
-    int masks[4];
-    float total_ms[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int cand = 0; cand < 4; ++cand) {
-        const int wide = ((cand & 1) ? (1 << TcUpGate) : 0) | ((cand & 2) ? (1 << TcDown) : 0);
-        masks[cand] = (base & ~fwd_bits) | wide;
-    }
+    const int fwd_bits = ((1 << TcUpGate) | (1 << TcDown)) * ((1 << kTcPairShift) | 1);
+    // candidates: each forward product on 128-row tiles, on 256-row tiles of one CTA, or on 256-row tiles of a
+    // CTA pair.  They are timed in interleaved rounds after a warm-up, so that the drift of the clocks under
+    // the power limit (a burst after idle, lower clocks later) does not favour whichever candidate runs first.
+    constexpr int kCand = 9;
+    int masks[kCand];
+    float total_ms[kCand] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    auto shape_bits = [](int shape, int kind) {
+        return shape == 2 ? ((1 << (kTcPairShift + kind)) | (1 << kind)) : (shape == 1 ? (1 << kind) : 0);
+    };
+    for (int cand = 0; cand < kCand; ++cand)
+        masks[cand] = (base & ~fwd_bits) | shape_bits(cand % 3, TcUpGate) | shape_bits(cand / 3, TcDown);
     auto run = [&](int reps) {
         for (int rep = 0; rep < reps && st == MODSE_OK; ++rep)
             st = modse_forward(layer, dtype, weights, x, n_tokens, y, workspace, workspace_bytes, save_for_backward,
                                cuda_stream);
     };
-    for (int cand = 0; cand < 4; ++cand) {          // warm-up: every candidate twice
+    for (int cand = 0; cand < kCand; ++cand) {      // warm-up: every candidate twice
         layer->tc.tile_mask = masks[cand];
         run(2);
     }
     for (int round = 0; round < 3 && st == MODSE_OK; ++round)
-        for (int cand = 0; cand < 4 && st == MODSE_OK; ++cand) {
+        for (int cand = 0; cand < kCand && st == MODSE_OK; ++cand) {
             layer->tc.tile_mask = masks[cand];
             float ms = 0.f;
             if (cudaEventRecord(ev[0], s) != cudaSuccess) st = MODSE_ERR_CUDA;
@@ -643,7 +645,7 @@ modse_status_t modse_tune_forward(modse_layer_t *layer, modse_dtype_t dtype, con
     int best_mask = base;
     if (st == MODSE_OK) {
         int best = 0;
-        for (int cand = 1; cand < 4; ++cand)
+        for (int cand = 1; cand < kCand; ++cand)
             if (total_ms[cand] < total_ms[best]) best = cand;
         best_mask = masks[best];
     }
@@ -677,7 +679,10 @@ void modse_debug_use_fma_path(int on) { tc_set_force_simt(on); }
 void modse_debug_set_default_tile_plan(int plan) { tc_set_default_plan(plan); }
 
 void modse_debug_set_dynamic_tiles(int on) { tc_set_dynamic_tiles(on); }
-void modse_debug_set_epilogue_warps(int mask_128, int mask_256) { tc_set_epilogue_warps16(mask_128, mask_256); }
+void modse_debug_set_epilogue_warps(int mask_128, int mask_256, int mask_pair)
+{
+    tc_set_epilogue_warps16(mask_128, mask_256, mask_pair);
+}
 
 void modse_debug_set_wait_limit_ms(int ms) { tc_set_wait_limit_ms(ms); }
 

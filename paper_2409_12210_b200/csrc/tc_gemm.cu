@@ -73,6 +73,7 @@ static int g_dynamic_tiles = 1;
 static int g_wait_limit_ms = 2000;
 static int g_skip_kind = -1, g_skip_tile = -1;
 static int g_epi16_narrow = 0, g_epi16_wide = kTcDefaultEpi16Wide;   // bit per product: sixteen epilogue warps
+static int g_epi16_pair = 0;
 
 bool tc_force_simt() { return g_force_simt != 0; }
 void tc_set_force_simt(int on) { g_force_simt = on ? 1 : 0; }
@@ -81,12 +82,12 @@ int tc_default_plan() { return g_default_plan; }
 void tc_set_dynamic_tiles(int on) { g_dynamic_tiles = on ? 1 : 0; }
 void tc_set_wait_limit_ms(int ms) { g_wait_limit_ms = ms < 1 ? 1 : (ms > 60000 ? 60000 : ms); }
 void tc_set_skip_tile(int kind, int tile) { g_skip_kind = kind; g_skip_tile = tile; }
-void tc_set_epilogue_warps16(int narrow_mask, int wide_mask)
+void tc_set_epilogue_warps16(int narrow_mask, int wide_mask, int pair_mask)
 {
-    g_epi16_narrow = narrow_mask & kTcPlanBits;
-    g_epi16_wide = wide_mask & kTcPlanBits;
+    g_epi16_narrow = narrow_mask & 63;
+    g_epi16_wide = wide_mask & 63;
+    g_epi16_pair = pair_mask & 63;
 }
-int tc_epilogue_warps(TcKind kind, bool wide) { return (((wide ? g_epi16_wide : g_epi16_narrow) >> (int)kind) & 1) ? 16 : 8; }
 
 namespace {
 
@@ -101,6 +102,7 @@ constexpr int kAccCols = 256;
 constexpr int kEpiRowBytes = 64;                 // a 32-element bf16 chunk of one row; 16-byte pieces XOR-swizzled
 constexpr int kEpiBufBytes = 32 * kEpiRowBytes;  // one warp's 32 rows: 2 KB
 template <int EPI> constexpr int epi_bytes() { return EPI * kEpiBufBytes; }   // one transposing buffer per epilogue warp
+constexpr int kMaxStages = 6;
 constexpr int kTileQ = 4;                        // tile indices in flight between the producer and the other roles
 
 // 128-row tiles: 4 stages of 16 KB rows + 32 KB columns.  256-row tiles: 3 stages of 2 x 16 KB rows + 32 KB columns.
@@ -135,7 +137,7 @@ struct TcParams {
 
 // control block behind the stages and the epilogue buffers
 struct SmemTail {
-    unsigned long long full[4], empty[4], tmem_full[2], tmem_empty[2], tq_full[kTileQ], tq_empty[kTileQ], tq_taken;
+    unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2], tq_full[kTileQ], tq_empty[kTileQ], tq_taken;
     unsigned int tmem_base;
     int abort_flag;
     int tile_q[kTileQ];
@@ -175,6 +177,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// the same test with acquire semantics at cluster scope: what the partner CTA wrote before its (release.cluster)
+// arrival is visible afterwards
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ unsigned long long global_ns()
 {
     unsigned long long t;
@@ -195,6 +211,23 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
     const unsigned long long t0 = global_ns();
     unsigned it = 0;
     while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 255u) == 0) {
+            if (*w.abort_flag || global_ns() - t0 > w.limit_ns) {
+                *w.abort_flag = 1;
+                atomicMax(w.status, kDevTimeout);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, const WaitCtx &w)
+{
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    unsigned it = 0;
+    while (!mbar_try_wait_cluster(bar, parity)) {
         if ((++it & 255u) == 0) {
             if (*w.abort_flag || global_ns() - t0 > w.limit_ns) {
                 *w.abort_flag = 1;
@@ -233,6 +266,23 @@ __device__ __forceinline__ void tma_load_rows(uint32_t dst, const CUtensorMap *m
     if (i < nboxes) tma_load_2d(dst + i * kBoxBytes, m64, bar, x, y + 64 * i);
 }
 
+// The same copies inside a pair of CTAs (cta_group::2): the data lands in the issuing CTA's shared memory, the
+// bytes are counted on a barrier of the pair's leader (`bar` is a shared::cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_rows_pair(uint32_t dst, const CUtensorMap *m64, const CUtensorMap *m128,
+                                                   uint32_t bar, int x, int y, int nboxes)
+{
+    int i = 0;
+    for (; i + 2 <= nboxes; i += 2) tma_load_2d_pair(dst + i * kBoxBytes, m128, bar, x, y + 64 * i);
+    if (i < nboxes) tma_load_2d_pair(dst + i * kBoxBytes, m64, bar, x, y + 64 * i);
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -248,6 +298,50 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+        : "memory");
+}
+// arrives on the barrier at the same shared-memory offset in both CTAs of the pair once the MMAs issued so far are done
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+// Arrival on a barrier of the partner CTA that also publishes what this thread wrote before it (release at
+// cluster scope).  Slow - of the order of a microsecond - so only the tile hand-out uses it.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Arrival on a barrier of either CTA of the pair that publishes nothing: what it signals (a tile index read, an
+// accumulator drained - ordered by the tcgen05 fence before it) is complete when the instruction issues.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
@@ -286,11 +380,11 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, bool mn_major)
     return (uint64_t)((saddr & 0x3FFFF) >> 4) | (lbo << 16) | (sbo << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128.
-__device__ __forceinline__ uint32_t make_idesc(bool a_mn, bool b_mn, int n)
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128 (one CTA) or 256 (a pair of CTAs).
+__device__ __forceinline__ uint32_t make_idesc(bool a_mn, bool b_mn, int n, int m = 128)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // Static hand-out (the global counter switched off): tiles are dealt to the CTAs in rounds of one tile each.
@@ -1158,6 +1252,310 @@ tc_grouped_gemm(const __grid_constant__ TcMaps maps, const __grid_constant__ TcP
     }
 }
 
+// ---------------------------------------------------------------------------
+// Two-CTA kernel (cta_group::2).  A cluster of two CTAs on neighbouring SMs
+// computes one 256-row tile with M = 256 instructions: each CTA stages its own
+// 128 rows of the row operand and HALF of the column operand (32 KB per k-block
+// instead of the 48 KB of the 128-row kernel, for the same MMA work per CTA), the
+// tensor cores of both SMs read both halves, and each CTA's tensor memory holds
+// the accumulator rows of its own half - 256 columns per tile, so two tiles fit
+// and the epilogue of one overlaps the main loop of the next, which a single CTA
+// cannot do for a 256-row tile.  The leader (cluster rank 0) issues the MMAs.
+//   full[s]        leader only: its producer posts the bytes of both CTAs, the
+//                  copies of both complete on it
+//   empty[s]       one per CTA; tcgen05.commit arrives on both
+//   tmem_full[a]   one per CTA; tcgen05.commit arrives on both
+//   tmem_empty[a]  leader only; one arrival per epilogue warp of both CTAs
+// Tiles come from the global counter through the leader's tile warp (or are dealt to the clusters round-robin).
+// ---------------------------------------------------------------------------
+constexpr int kPairStages = 6;
+constexpr int kPairHalfB = 2 * kBoxBytes;                     // this CTA's half of the column operand: up to 128 x 64
+constexpr int kPairStageBytes = kARegion + kPairHalfB;        // 32 KB
+template <int EPI> constexpr size_t pair_smem_bytes()
+{
+    return 1024 + (size_t)kPairStages * kPairStageBytes + epi_bytes<EPI>() + sizeof(SmemTail);
+}
+static_assert(pair_smem_bytes<kMaxEpiWarps>() <= 232448, "shared memory per CTA");
+static_assert(kPairStages <= kMaxStages, "barrier arrays");
+
+// Accumulator columns of a pair tile (each CTA stages half of them): a multiple of 128, so that a half is whole
+// 64-column boxes; columns past the tile's own are computed from whatever lies beside them and never stored.
+template <int KIND>
+__device__ __forceinline__ int pair_n_mma(const Tile &t)
+{
+    if constexpr (KIND == TcUpGate) return 2 * t.ncols;       // gate columns in the leader, up columns in its partner
+    else return (t.ncols + 127) & ~127;
+}
+
+// This CTA's half of the column operand of k-block kb.
+template <int KIND>
+__device__ __forceinline__ void load_cols_pair(const TcMaps &maps, const Tile &t, int rank, int kb, uint32_t dst, uint32_t bar)
+{
+    const int half = pair_n_mma<KIND>(t) / 2, nb = half / 64;
+    if constexpr (KIND == TcUpGate) {
+        if (rank == 0) tma_load_rows_pair(dst, &maps.wgate, &maps.wgate128, bar, kb * 64, t.ho + t.n0, nb);
+        else tma_load_rows_pair(dst, &maps.wup, &maps.wup128, bar, kb * 64, t.ho + t.n0, nb);
+    } else if constexpr (KIND == TcDown) {
+        tma_load_rows_pair(dst, &maps.wdown, &maps.wdown128, bar, t.ho + kb * 64, t.n0 + rank * half, nb);
+    } else if constexpr (KIND == TcDownDgrad) {
+        for (int i = 0; i < nb; ++i)
+            tma_load_2d_pair(dst + i * kBoxBytes, &maps.wdown, bar, t.ho + t.n0 + rank * half + 64 * i, kb * 64);
+    } else if constexpr (KIND == TcDownWgrad) {
+        for (int i = 0; i < nb; ++i)
+            tma_load_2d_pair(dst + i * kBoxBytes, &maps.hm, bar, 0, t.pbase + ((t.n0 + rank * half) / 64 + i) * t.cp + kb * 64);
+    } else if constexpr (KIND == TcUpGateDgrad) {
+        const int hk = t.h / 64;
+        const bool second = kb >= hk;
+        const int kk = second ? kb - hk : kb;
+        const CUtensorMap *bm = second ? &maps.wup : &maps.wgate;
+        for (int i = 0; i < nb; ++i) tma_load_2d_pair(dst + i * kBoxBytes, bm, bar, t.n0 + rank * half + 64 * i, t.ho + kk * 64);
+    } else {
+        for (int i = 0; i < nb; ++i)
+            tma_load_2d_pair(dst + i * kBoxBytes, &maps.xp, bar, t.n0 + rank * half + 64 * i, t.prow0 + kb * 64);
+    }
+}
+
+// This CTA's 128 rows of the row operand of k-block kb (t: this CTA's half of the tile).
+template <int KIND>
+__device__ __forceinline__ void load_rows_pair(const TcMaps &maps, const Tile &t, int kb, uint32_t dst, uint32_t bar)
+{
+    if constexpr (KIND == TcUpGate) {
+        tma_load_rows_pair(dst, &maps.xp, &maps.xp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
+    } else if constexpr (KIND == TcDown) {
+        tma_load_rows_pair(dst, &maps.hm, &maps.hm128, bar, 0, t.pbase + kb * t.cp + t.m0, t.a_boxes);
+    } else if constexpr (KIND == TcDownDgrad) {
+        tma_load_rows_pair(dst, &maps.dyp, &maps.dyp128, bar, kb * 64, t.prow0 + t.m0, t.a_boxes);
+    } else if constexpr (KIND == TcDownWgrad) {
+        for (int i = 0; i < t.a_boxes; ++i) tma_load_2d_pair(dst + i * kBoxBytes, &maps.dyp, bar, t.m0 + 64 * i, t.prow0 + kb * 64);
+    } else if constexpr (KIND == TcUpGateDgrad) {
+        const int hk = t.h / 64;
+        const bool second = kb >= hk;
+        const int kk = second ? kb - hk : kb;
+        tma_load_rows_pair(dst, second ? &maps.db : &maps.da, second ? &maps.db128 : &maps.da128, bar, 0,
+                           t.pbase + kk * t.cp + t.m0, t.a_boxes);
+    } else {
+        const CUtensorMap *am = t.which ? &maps.db : &maps.da;
+        for (int i = 0; i < t.a_boxes; ++i)
+            tma_load_2d_pair(dst + i * kBoxBytes, am, bar, 0, t.pbase + (t.m0 / 64 + i) * t.cp + kb * 64);
+    }
+}
+
+// Tile hand-out inside a pair: the leader's tile warp takes tile after tile from the global counter and writes
+// each index into the queue slot of both CTAs (its partner's through the cluster's shared address space, the
+// arrival that follows releases it at cluster scope); every consuming role of either CTA frees the slot on the
+// leader's barrier.  Consumers: the leader's TMA, MMA and epilogue warps, its partner's TMA and epilogue warps.
+
+__device__ __forceinline__ void hand_out_tiles_pair(const TcParams &prm, SmemTail *st, int total, const WaitCtx &w)
+{
+    for (int it = 0;; ++it) {
+        const int slot = it & (kTileQ - 1);
+        const uint32_t ph = (uint32_t)(it / kTileQ) & 1u;
+        if (it > 0 && !mbar_wait(smem_u32(&st->tq_taken), (uint32_t)(it - 1) & 1u, w)) return;
+        if (!mbar_wait_cluster(smem_u32(&st->tq_empty[slot]), ph ^ 1u, w)) return;
+        int tile = atomicAdd(prm.tile_counter, 1);
+        if (tile >= total) tile = -1;
+        st->tile_q[slot] = tile;
+        asm volatile("st.shared::cluster.b32 [%0], %1;" ::"r"(map_to_cta(smem_u32(&st->tile_q[slot]), 1)), "r"(tile) : "memory");
+        mbar_arrive(smem_u32(&st->tq_full[slot]));
+        mbar_arrive_cluster(map_to_cta(smem_u32(&st->tq_full[slot]), 1));
+        if (tile < 0) return;
+    }
+}
+
+// The it-th tile of this cluster (-1: no more), not yet released.
+template <int KIND>
+__device__ __forceinline__ int peek_tile_pair(const TcParams &prm, SmemTail *st, int it, int total, int cluster_id,
+                                              int n_clusters, const WaitCtx &w, bool &ok)
+{
+    if (!prm.dynamic) {
+        const int tile = dealt_tile<KIND>(it, cluster_id, n_clusters);
+        return tile >= total ? -1 : tile;
+    }
+    const int slot = it & (kTileQ - 1);
+    const uint32_t ph = (uint32_t)(it / kTileQ) & 1u;
+    if (!mbar_wait_cluster(smem_u32(&st->tq_full[slot]), ph, w)) { ok = false; return -1; }
+    return *reinterpret_cast<volatile int *>(&st->tile_q[slot]);
+}
+__device__ __forceinline__ void release_tile_pair(const TcParams &prm, SmemTail *st, int it)
+{
+    if (prm.dynamic) mbar_arrive_remote(map_to_cta(smem_u32(&st->tq_empty[it & (kTileQ - 1)]), 0));
+}
+
+template <int KIND, int VAR, int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(threads_of<EPI>(), 1)
+tc_grouped_gemm_pair(const __grid_constant__ TcMaps maps, const __grid_constant__ TcParams prm)
+{
+    constexpr int NQ = EPI / 4;
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t pad = ((raw + 1023u) & ~1023u) - raw;
+    unsigned char *smem = smem_raw + pad;
+    const uint32_t stage_base = raw + pad;
+    unsigned char *epi_bufs = smem + (size_t)kPairStages * kPairStageBytes;
+    SmemTail *st = reinterpret_cast<SmemTail *>(epi_bufs + EPI * kEpiBufBytes);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int rank = (int)cluster_ctarank();
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+    if (tid == 0) {
+        for (int s = 0; s < kPairStages; ++s) {
+            mbar_init(smem_u32(&st->full[s]), 1);
+            mbar_init(smem_u32(&st->empty[s]), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&st->tmem_full[a]), 1);
+            mbar_init(smem_u32(&st->tmem_empty[a]), 2 * EPI);      // one lane of every epilogue warp of both CTAs
+        }
+        mbar_init(smem_u32(&st->tq_taken), 1);
+        for (int q = 0; q < kTileQ; ++q) {
+            mbar_init(smem_u32(&st->tq_full[q]), 1);
+            mbar_init(smem_u32(&st->tq_empty[q]), 3 + 2 * EPI);   // used in the leader only
+        }
+        st->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    build_schedule<KIND, true>(prm, st, reinterpret_cast<int *>(epi_bufs), reinterpret_cast<int *>(epi_bufs) + kMaxExperts, tid);
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&st->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                 // both CTAs' barriers exist before any remote arrival or copy completion
+    tc_fence_after();
+    const uint32_t tmem_base = st->tmem_base;
+    const int total_tiles = st->tstart[prm.meta.N];
+    const WaitCtx wc{&st->abort_flag, prm.status, prm.wait_limit_ns};
+
+    if (warp == 0) {
+        // ===================== TMA producer (both CTAs) =====================
+        if (lane == 0) {
+            int stage = 0, cursor = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (int it = 0; ok; ++it) {
+                const int tile = peek_tile_pair<KIND>(prm, st, it, total_tiles, cluster_id, n_clusters, wc, ok);
+                if (!ok) break;
+                release_tile_pair(prm, st, it);
+                if (prm.dynamic && rank == 0) mbar_arrive(smem_u32(&st->tq_taken));
+                if (tile < 0 || tile == prm.skip_tile) break;
+                const Tile t0 = decode_tile<KIND, true>(prm, st, tile, cursor);
+                const Tile mine = rank ? second_half(t0) : t0;
+                const uint32_t bytes =
+                    (uint32_t)(t0.a_boxes + t0.a_boxes_peer + 2 * (pair_n_mma<KIND>(t0) / 128)) * kBoxBytes;
+                for (int kb = 0; kb < t0.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->empty[stage]), phase ^ 1u, wc)) { ok = false; break; }
+                    const uint32_t leader_bar = map_to_cta(smem_u32(&st->full[stage]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(smem_u32(&st->full[stage]), bytes);
+                    const uint32_t a_dst = stage_base + stage * kPairStageBytes;
+                    load_rows_pair<KIND>(maps, mine, kb, a_dst, leader_bar);
+                    load_cols_pair<KIND>(maps, t0, rank, kb, a_dst + kARegion, leader_bar);
+                    ++issued;
+                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok && rank == 0) {
+                // the copies of both CTAs complete on the leader's barriers: it lets those in flight land
+                const int n = issued < kPairStages ? (int)issued : kPairStages;
+                for (int i = 1; i <= n; ++i) {
+                    int s2 = stage - i;
+                    uint32_t ph = phase;
+                    if (s2 < 0) { s2 += kPairStages; ph ^= 1u; }
+                    const unsigned long long tb = global_ns();
+                    while (!mbar_try_wait(smem_u32(&st->full[s2]), ph) && global_ns() - tb < prm.wait_limit_ns) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ===================== MMA issuer (leader only) =====================
+        if (lane == 0 && rank == 0) {
+            int stage = 0, cursor = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            constexpr bool a_mn = KindTraits<KIND>::a_mn, b_mn = KindTraits<KIND>::b_mn;
+            constexpr uint32_t a_step = a_mn ? (2048u >> 4) : (32u >> 4);
+            constexpr uint32_t b_step = b_mn ? (2048u >> 4) : (32u >> 4);
+            for (int it = 0; ok; ++it) {
+                const int tile = peek_tile_pair<KIND>(prm, st, it, total_tiles, cluster_id, n_clusters, wc, ok);
+                if (!ok) break;
+                release_tile_pair(prm, st, it);
+                if (tile < 0) break;
+                const Tile t = decode_tile<KIND, true>(prm, st, tile, cursor);
+                const int acc = it & 1;
+                const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&st->tmem_empty[acc]), acc_phase ^ 1u, wc)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t tacc = tmem_base + (uint32_t)(acc * kAccCols);
+                const uint32_t idesc = make_idesc(a_mn, b_mn, pair_n_mma<KIND>(t), 256);
+                for (int kb = 0; kb < t.nk; ++kb) {
+                    if (!mbar_wait(smem_u32(&st->full[stage]), phase, wc)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = stage_base + stage * kPairStageBytes;
+                    const uint64_t adesc = make_desc(a_addr, a_mn);
+                    const uint64_t bdesc = make_desc(a_addr + kARegion, b_mn);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        umma_bf16_pair(tacc, adesc + (uint64_t)(ks * a_step), bdesc + (uint64_t)(ks * b_step), idesc,
+                                       (kb > 0 || ks > 0) ? 1u : 0u);
+                    umma_commit_pair(smem_u32(&st->empty[stage]));
+                    if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (t.nk > 0) {
+                    umma_commit_pair(smem_u32(&st->tmem_full[acc]));
+                } else {
+                    mbar_arrive(smem_u32(&st->tmem_full[acc]));
+                    mbar_arrive_cluster(map_to_cta(smem_u32(&st->tmem_full[acc]), 1));
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ===================== tile hand-out (leader only) =====================
+        if (lane == 0 && rank == 0 && prm.dynamic) hand_out_tiles_pair(prm, st, total_tiles, wc);
+    } else if (warp >= kFirstEpiWarp) {
+        // ===================== epilogue (both CTAs) =====================
+        const int quad = warp & 3;
+        const int cq = (warp - kFirstEpiWarp) >> 2;
+        const int row = quad * 32 + lane;
+        unsigned char *stg = epi_bufs + (warp - kFirstEpiWarp) * kEpiBufBytes;
+        const uint32_t leader_empty0 = map_to_cta(smem_u32(&st->tmem_empty[0]), 0);
+        const uint32_t leader_empty1 = map_to_cta(smem_u32(&st->tmem_empty[1]), 0);
+        int cursor = 0;
+        bool ok = true;
+        for (int it = 0; ok; ++it) {
+            const int tile = peek_tile_pair<KIND>(prm, st, it, total_tiles, cluster_id, n_clusters, wc, ok);
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) release_tile_pair(prm, st, it);
+            if (tile < 0) break;
+            const Tile t0 = decode_tile<KIND, true>(prm, st, tile, cursor);
+            const Tile mine = rank ? second_half(t0) : t0;
+            const int acc = it & 1;
+            const uint32_t acc_phase = (uint32_t)(it >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&st->tmem_full[acc]), acc_phase, wc)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t tacc = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kAccCols);
+            if (mine.mrows > 0) epilogue_row<KIND, VAR, NQ>(prm, mine, tacc, row, lane, cq, stg);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_remote(acc ? leader_empty1 : leader_empty0);
+        }
+    }
+
+    // ---- teardown: neither CTA leaves while its partner may still touch its shared or tensor memory ----
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
 // Sums the partial row dots of the down dgrad in slot order and divides by the gate:
 // dg[t, j] = <dY_t W_down, Hm_row> / g = <dY_t, E_(t,j)>.  One thread per assignment.
 __global__ void __launch_bounds__(256)
@@ -1282,6 +1680,38 @@ cudaError_t launch_kind(const TcMaps &maps, const TcParams &prm, int grid, bool 
                 : launch_epi<KIND, false, 0>(maps, prm, grid, epi, s, launches);
 }
 
+template <int KIND, int VAR, int EPI>
+cudaError_t launch_pair_one(const TcMaps &maps, const TcParams &prm, int grid, cudaStream_t s, int *launches)
+{
+    auto kern = tc_grouped_gemm_pair<KIND, VAR, EPI>;
+    constexpr size_t smem = pair_smem_bytes<EPI>();
+    static unsigned long long attr_done = 0;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev > 63 || !((attr_done >> dev) & 1ull)) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev <= 63) attr_done |= 1ull << dev;
+    }
+    kern<<<grid & ~1, threads_of<EPI>(), smem, s>>>(maps, prm);     // whole clusters of two
+    e = cudaGetLastError();
+    if (e == cudaSuccess && launches) ++*launches;
+    return e;
+}
+
+template <int KIND, bool HAS_VAR>
+cudaError_t launch_pair(const TcMaps &maps, const TcParams &prm, int grid, int var, int epi, cudaStream_t s, int *launches)
+{
+    if constexpr (HAS_VAR) {
+        if (var)
+            return epi == 16 ? launch_pair_one<KIND, 1, 16>(maps, prm, grid, s, launches)
+                             : launch_pair_one<KIND, 1, 8>(maps, prm, grid, s, launches);
+    }
+    return epi == 16 ? launch_pair_one<KIND, 0, 16>(maps, prm, grid, s, launches)
+                     : launch_pair_one<KIND, 0, 8>(maps, prm, grid, s, launches);
+}
+
 int sm_count(TcPlan &plan)
 {
     if (plan.sm_count == 0) {
@@ -1333,8 +1763,20 @@ cudaError_t tc_launch(TcPlan &plan, TcKind kind, const TcMaps &maps, const Layer
     const int grid = sm_count(plan);
     const int mask = plan.tile_mask >= 0 ? plan.tile_mask : tc_default_plan();
     const bool wide = ((mask >> (int)kind) & 1) != 0;
-    const int epi = tc_epilogue_warps(kind, wide);
+    // the two-CTA kernel has no row-gathering loads: the fused up/gate product stays on one CTA
+    const bool pair = ((mask >> (kTcPairShift + (int)kind)) & 1) != 0 && grid >= 2 && !(kind == TcUpGate && (fuse & kFuseGather));
+    const int epi = (((pair ? g_epi16_pair : wide ? g_epi16_wide : g_epi16_narrow) >> (int)kind) & 1) ? 16 : 8;
     cudaError_t e = cudaErrorInvalidValue;
+    if (pair) {
+        switch (kind) {
+        case TcUpGate: e = launch_pair<TcUpGate, false>(maps, prm, grid, 0, epi, s, launches); break;
+        case TcDown: e = launch_pair<TcDown, true>(maps, prm, grid, fuse & kFuseScatter, epi, s, launches); break;
+        case TcDownDgrad: e = launch_pair<TcDownDgrad, true>(maps, prm, grid, fuse & kFuseDgRowdot, epi, s, launches); break;
+        case TcDownWgrad: e = launch_pair<TcDownWgrad, false>(maps, prm, grid, 0, epi, s, launches); break;
+        case TcUpGateDgrad: e = launch_pair<TcUpGateDgrad, true>(maps, prm, grid, fuse & kFuseScatter, epi, s, launches); break;
+        case TcUpGateWgrad: e = launch_pair<TcUpGateWgrad, false>(maps, prm, grid, 0, epi, s, launches); break;
+        }
+    } else
     switch (kind) {
     case TcUpGate: e = launch_kind<TcUpGate, true>(maps, prm, grid, wide, fuse & kFuseGather, epi, s, launches); break;
     case TcDown: e = launch_kind<TcDown, true>(maps, prm, grid, wide, fuse & kFuseScatter, epi, s, launches); break;

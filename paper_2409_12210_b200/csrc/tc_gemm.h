@@ -17,12 +17,20 @@ enum TcKind : int {
     TcUpGateWgrad = 5   // dWg = dA^T xp, dWu = dB^T xp
 };
 
-// Tile plan: bit k set = product kind k runs on 256-row tiles (two 128-row halves that share the column
-// operand), clear = on 128-row tiles with two accumulators in flight.  Default: the four products with
-// long K loops (down, down wgrad, up/gate dgrad, up/gate wgrad) on 256-row tiles.
-constexpr int kTcDefaultPlan = (1 << TcDown) | (1 << TcDownWgrad) | (1 << TcUpGateDgrad) | (1 << TcUpGateWgrad);
-constexpr int kTcPlanBits = 63;
-// Epilogue warps per CTA: bit k set = product k runs sixteen of them on its 256-row tiles (eight otherwise).
+// Tile plan: one of three kernel shapes per product kind k.
+//   bit 8 + k set : 256-row tiles computed by a pair of CTAs on neighbouring SMs (each stages its own 128 rows
+//                   and half of the column operand; two tiles' accumulators fit, so epilogues overlap main loops);
+//   else bit k set: 256-row tiles computed by one CTA (two 128-row halves that share the column operand; both
+//                   accumulators belong to the tile);
+//   else          : 128-row tiles, two accumulators in flight.
+// Default: every product on CTA pairs; the low bits say what a product falls back to where the pair kernel does
+// not apply (the row-gathering up/gate product, a device with a single SM).
+constexpr int kTcPairShift = 8;
+constexpr int kTcOneCtaDefault = (1 << TcDown) | (1 << TcDownWgrad) | (1 << TcUpGateDgrad) | (1 << TcUpGateWgrad);
+constexpr int kTcDefaultPlan = (63 << kTcPairShift) | kTcOneCtaDefault;
+constexpr int kTcPlanBits = (63 << kTcPairShift) | 63;
+// Epilogue warps per CTA: bit k set = product k runs sixteen of them on its one-CTA 256-row tiles (eight
+// otherwise): that shape cannot overlap its epilogue with the next main loop, so more warps shorten what is exposed.
 constexpr int kTcDefaultEpi16Wide = (1 << TcUpGate) | (1 << TcDownDgrad);
 
 // Optional fusions across the permutation (what lies either side of the permute / un-permute steps).
@@ -69,8 +77,8 @@ void tc_set_default_plan(int mask);   // tile plan used by layers that have none
 int tc_default_plan();
 void tc_set_dynamic_tiles(int on);    // 1 (default): CTAs take tiles from a shared counter; 0: tiles are dealt statically
 void tc_set_wait_limit_ms(int ms);    // limit of every bounded wait inside the kernels (default 2000)
-void tc_set_epilogue_warps16(int narrow_mask, int wide_mask);   // bit per product: sixteen epilogue warps on 128- / 256-row tiles
-int tc_epilogue_warps(TcKind kind, bool wide);
+// bit per product: sixteen epilogue warps on 128-row tiles / one-CTA 256-row tiles / CTA-pair tiles
+void tc_set_epilogue_warps16(int narrow_mask, int wide_mask, int pair_mask);
 void tc_set_skip_tile(int kind, int tile);   // the producer of the CTA that gets `tile` of product `kind` stops there (-1: off)
 
 bool tc_fill_maps(TcMaps &maps, const LayerMeta &m, const WsLayout &L, const WsPtrs &p, const modse_weights_t *w,

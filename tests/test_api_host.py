@@ -111,7 +111,9 @@ def test_tile_plan_validation_needs_no_gpu():
     assert layer.tile_plan() == B.DEFAULT_TILE_PLAN
     layer.set_tile_plan(-1)
     assert layer.tile_plan() == -1
-    for bad in (-2, 0x100, 0x40):
+    layer.set_tile_plan(0x3F3F)
+    assert layer.tile_plan() == 0x3F3F
+    for bad in (-2, 0x4000, 0x40, 0x80):
         with pytest.raises(B.ModseError) as ei:
             layer.set_tile_plan(bad)
         assert ei.value.status == B.MODSE_ERR_INVALID_ARG

@@ -20,6 +20,7 @@ def lib():
     yield
     B.debug_set_wait_limit_ms(2000)
     B.debug_skip_tile_loads(-1, -1)
+    B.debug_set_default_tile_plan(B.DEFAULT_TILE_PLAN)
 
 
 def setup_layer(inp, save, slack_bytes=0):
@@ -35,15 +36,18 @@ def setup_layer(inp, save, slack_bytes=0):
     return layer, w, x, y, ws
 
 
+@pytest.mark.parametrize("plan", [0x3F3A, 0b111010], ids=["cta_pairs", "one_cta"])
 @pytest.mark.parametrize("product", [0, 1])
-def test_a_wait_that_runs_out_is_reported_and_the_gpu_stays_usable(product):
-    """The producer of one CTA is told to load nothing for its first tile: no copy and no MMA of that CTA is in
-    flight, its MMA warp waits for data that never comes, gives up after the (shortened) limit, the CTA frees
-    its tensor memory and the kernel returns.  The host reads the time-out, and the next forward is correct."""
+def test_a_wait_that_runs_out_is_reported_and_the_gpu_stays_usable(product, plan):
+    """The producer of one CTA (of both CTAs of a pair) is told to load nothing for its first tile: no copy and no
+    MMA of that CTA is in flight, its MMA warp waits for data that never comes, gives up after the (shortened)
+    limit, the CTA frees its tensor memory and the kernel returns.  The host reads the time-out, and the next
+    forward is correct."""
     import torch
     from paper_2409_12210_b200 import binding as B
     inp, _ = H.screened(TINY_BF16)
     layer, w, x, y, ws = setup_layer(inp, save=False)
+    B.debug_set_default_tile_plan(plan)
     B.debug_set_wait_limit_ms(50)
     B.debug_skip_tile_loads(product, 0)
     try:
@@ -58,6 +62,7 @@ def test_a_wait_that_runs_out_is_reported_and_the_gpu_stays_usable(product):
     ora = H.run_oracle(inp, backward=False)
     assert H.rel_err_beyond_storage(y.float().cpu().numpy(), ora["y"]) <= 2e-2
     layer.destroy()
+    B.debug_set_default_tile_plan(B.DEFAULT_TILE_PLAN)
 
 
 @pytest.mark.parametrize("fuse", [0, 2])

@@ -28,7 +28,7 @@ def lib():
 
 
 @pytest.mark.parametrize("cfg", CASES, ids=lambda c: c.name)
-@pytest.mark.parametrize("plan", [0, 63])
+@pytest.mark.parametrize("plan", [0, 63, 0x3F00])
 def test_gathering_up_gate_product_gives_the_same_bits(cfg, plan):
     from paper_2409_12210_b200 import binding as B
     inp, _ = H.screened(cfg)
@@ -49,7 +49,7 @@ def test_gathering_up_gate_product_gives_the_same_bits(cfg, plan):
 
 
 @pytest.mark.parametrize("cfg", CASES, ids=lambda c: c.name)
-@pytest.mark.parametrize("plan", [0, 63])
+@pytest.mark.parametrize("plan", [0, 63, 0x3F00])
 def test_gate_gradient_from_the_down_dgrad_epilogue(cfg, plan):
     from paper_2409_12210_b200 import binding as B
     inp, _ = H.screened(cfg)
@@ -69,7 +69,7 @@ def test_gate_gradient_from_the_down_dgrad_epilogue(cfg, plan):
 
 
 @pytest.mark.parametrize("cfg", CASES, ids=lambda c: c.name)
-@pytest.mark.parametrize("plan", [0, 63])
+@pytest.mark.parametrize("plan", [0, 63, 0x3F00])
 def test_scatter_adding_epilogues_give_the_same_bits_as_the_combine_kernels(cfg, plan):
     from paper_2409_12210_b200 import binding as B
     inp, _ = H.screened(cfg)

@@ -197,18 +197,26 @@ def test_bf16_results_are_bitwise_reproducible_and_independent_of_tile_shape_and
     try:
         B.debug_set_default_tile_plan(0)               # 128-row tiles everywhere
         c = H.run_gpu(inp, True)
-        B.debug_set_default_tile_plan(63)              # 256-row tiles everywhere
+        B.debug_set_default_tile_plan(63)              # 256-row tiles of one CTA everywhere
         e = H.run_gpu(inp, True)
+        B.debug_set_default_tile_plan(63 << B.PAIR_SHIFT)   # 256-row tiles of a CTA pair everywhere
+        p = H.run_gpu(inp, True)
+        B.debug_set_epilogue_warps(63, 63, 63)         # sixteen epilogue warps in every kernel
+        B.debug_set_default_tile_plan(0b101010 | (0b010101 << B.PAIR_SHIFT))   # the shapes mixed
+        q = H.run_gpu(inp, True)
         B.debug_set_default_tile_plan(B.DEFAULT_TILE_PLAN)
         B.debug_set_dynamic_tiles(False)               # tiles dealt round-robin instead of taken from the counter
         f = H.run_gpu(inp, True)
     finally:
         B.debug_set_default_tile_plan(B.DEFAULT_TILE_PLAN)
         B.debug_set_dynamic_tiles(True)
+        B.debug_set_epilogue_warps()
     for k in ("y", "dx", "dw_router", "dw_gate", "dw_up", "dw_down", "dg", "dz"):
         assert np.array_equal(a[k], b[k]), k
         assert np.array_equal(a[k], c[k]), k
         assert np.array_equal(a[k], e[k]), k
+        assert np.array_equal(a[k], p[k]), k
+        assert np.array_equal(a[k], q[k]), k
         assert np.array_equal(a[k], f[k]), k
 
 
@@ -229,7 +237,7 @@ def test_tuned_plan_gives_identical_results():
     layer.forward(wr, wg, wu, wd, x, y0, ws, True)
     assert layer.tile_plan() == -1
     plan = layer.tune_forward(wr, wg, wu, wd, x, y1, ws, True)
-    assert plan >= 0 and (plan & ~63) == 0 and layer.tile_plan() == plan
+    assert plan >= 0 and (plan & ~0x3F3F) == 0 and layer.tile_plan() == plan
     assert torch.equal(y0, y1)
     dx = torch.empty_like(x); dwr = torch.empty(wr.shape, dtype=torch.float32, device=dev)
     dwg, dwu, dwd = (torch.empty_like(w) for w in (wg, wu, wd))
