@@ -37,13 +37,14 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 NOMINAL_BF16_DENSE_TFLOPS = 2250.0     # vendor figure for dense bf16, the "bf16 dense peak" of the target
 NOMINAL_HBM_GBS = 8000.0               # "~8 TB/s"
 BURST_REGION_S = 1.0                   # timed regions shorter than this run on burst clocks: burst peak applies
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-# profiles/tc_grouped_gemm_train_16k_ncu_full.md; valid only for that workload and for the kernel source it was
-# taken from (first 16 hex digits of the SHA-256 of csrc/tc_gemm.cu), otherwise "traffic" is reported as null.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised in
+# profiles/tc_grouped_gemm_pair_train_16k_ncu.md (one kernel and one launch per ncu run, --clock-control none);
+# valid only for that workload, for the library's default tile plan and for the kernel source they were taken
+# from (first 16 hex digits of the SHA-256 of csrc/tc_gemm.cu), otherwise "traffic" is reported as null.
 NCU_TRAFFIC = {
-    "workload": "train_16k", "tc_gemm_sha256_16": "c818e5c311c654cd",
-    "bytes_per_launch": {"upgate_gemm_swiglu": 1.591e9, "down_gemm": 0.932e9, "down_dgrad_swiglu_bwd": 1.953e9,
-                         "down_wgrad": 0.753e9, "upgate_dgrad": 1.910e9, "upgate_wgrad": 1.310e9},
+    "workload": "train_16k", "tc_gemm_sha256_16": "66fa88c46baa70c4",
+    "bytes_per_launch": {"upgate_gemm_swiglu": 1.589e9, "down_gemm": 0.948e9, "down_dgrad_swiglu_bwd": 1.831e9,
+                         "down_wgrad": 0.686e9, "upgate_dgrad": 1.910e9, "upgate_wgrad": 1.242e9},
 }
 
 

@@ -62,8 +62,8 @@ modse_status_t modse_last_create_error(void); /* per calling thread */
 modse_status_t modse_destroy(modse_layer_t *layer); /* NULL is accepted */
 
 /* Sec. 3.1, Eq. 5-6: returns 1 iff n_experts is even and every adjacent pair
- * (2p, 2p+1) - "expert 0 and expert 1 on the same GPU, and so forth",
- * Sec. 3.2 - has the same width sum 2h; *pair_sum_out (may be NULL) gets it.  */
+ * (2p, 2p+1) - the pairs that the expert-pair allocation of Sec. 3.2 places on
+ * one GPU each - has the same width sum 2h; *pair_sum_out (may be NULL) gets it. */
 int modse_check_pairs(const int *ffn_sizes, int n_experts, int *pair_sum_out);
 
 const char *modse_status_string(modse_status_t status);
