@@ -13,10 +13,13 @@
 //                      that the sum is rounded to the layer type only once.)
 //   dg_permute_kernel  dg[t,j] = <dY_t, E_(t,j)>, rows of dY in group order.
 //   router_dx_kernel   softmax Jacobian on the kept logits and dx assembly.
-//   router_dwr_kernel  per-block partial sums of dW_router = dz^T x, reduced in a
-//                      fixed order by reduce_dwr_kernel (reproducible).
+//   router_dwr_kernel  per-block partial sums of dW_router = dz^T x (fp32 FMA), for bf16
+//   router_dwr_mma_kernel  layers on tensor cores; reduced in a fixed order by
+//                      reduce_dwr_kernel (reproducible).
 //
 // No kernel uses a floating-point atomic; every sum has a fixed order.
+#include <algorithm>
+
 #include "modse_internal.h"
 
 namespace modse {
@@ -979,6 +982,142 @@ router_dwr_kernel(const T *__restrict__ x, int Ttok, int d, int N, int k, const 
     }
 }
 
+// ---------------------------------------------------------------------------
+// The same partial sums for bf16 layers on tensor cores (mma.sync m16n8k16): dW[e, c] = sum_t dz[t, e] x[t, c]
+// is a [8 experts x 64 tokens] . [64 tokens x columns] product per token block.  dz is fp32: it enters as the
+// sum of two bf16 numbers, hi = bf16(dz) in rows 0-7 of the A operand and lo = bf16(dz - hi) in rows 8-15, so one
+// instruction forms both parts (x is bf16, every product is exact in fp32) and the two halves of the
+// accumulator are added at the end; what is lost is below 2^-17 of each term.  A warp owns a unit of 64 tokens x
+// 256 columns: it stages 32 columns at a time in shared memory (16-byte loads, rows padded to 80 bytes) and reads
+// them back transposed with ldmatrix, which yields the B operand (pairs of consecutive tokens per column).  Units
+// are dealt to the blocks round-robin, so every SM gets the same number of them (+-1).
+// ---------------------------------------------------------------------------
+constexpr int kDwrUnitCols = 256;
+constexpr int kDwrChunkCols = 32;
+constexpr int kDwrXPitch = 80;                       // bytes per staged row: 64 of data + 16 of skew (conflict-free ldmatrix)
+constexpr int kDwrZPitch = 72;                       // bf16 per expert row of the dz slice: 64 tokens + 8 of skew
+constexpr int kDwrWarpSmem = kDwrTokB * kDwrXPitch + 2 * 8 * kDwrZPitch * 2;   // x chunk + hi and lo slices of dz
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+
+__global__ void __launch_bounds__(256)
+router_dwr_mma_kernel(const __nv_bfloat16 *__restrict__ x, int Ttok, int d, int N, int k, const int *__restrict__ topk_idx,
+                      const float *__restrict__ dz, float *__restrict__ dwr_partial, const float *__restrict__ logits,
+                      const int *__restrict__ counts_slot, float aux_scale, const float *__restrict__ dense, int nblk,
+                      int nslice)
+{
+    extern __shared__ __align__(16) unsigned char dwr_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, tq = lane & 3;
+    unsigned char *xs = dwr_smem + (size_t)warp * kDwrWarpSmem;
+    __nv_bfloat16 *zh = reinterpret_cast<__nv_bfloat16 *>(xs + kDwrTokB * kDwrXPitch);      // [8][kDwrZPitch]
+    __nv_bfloat16 *zl = zh + 8 * kDwrZPitch;
+    const uint32_t xs_addr = (uint32_t)__cvta_generic_to_shared(xs);
+    const int units = nblk * nslice;
+    const float inv_T = 1.0f / (float)Ttok;
+    for (int u = blockIdx.x + gridDim.x * warp; u < units; u += gridDim.x * 8) {
+        const int blk = u / nslice, slice = u - blk * nslice;
+        const int t0 = blk * kDwrTokB;
+        const int ntok = min(kDwrTokB, Ttok - t0);
+        const int c_begin = slice * kDwrUnitCols, c_end = min(d, c_begin + kDwrUnitCols);
+        for (int g0 = 0; g0 < N; g0 += 8) {
+            // this group's slice of dz (dense over its 8 experts), split into hi and lo: a lane builds tokens lane, lane + 32
+            __syncwarp();
+            for (int tl = lane; tl < kDwrTokB; tl += 32) {
+                float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                if (tl < ntok) {
+                    const int t = t0 + tl;
+                    if (dense != nullptr) {
+                        for (int i = 0; i < 8; ++i)
+                            if (g0 + i < N) v[i] = dense[(size_t)t * N + g0 + i];
+                    } else {
+                        for (int j = 0; j < k; ++j) {
+                            const int e = topk_idx[(size_t)t * k + j] - g0;
+                            const float dzv = dz[(size_t)t * k + j];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                if (e == i) v[i] = dzv;
+                        }
+                        if (aux_scale != 0.f) {
+                            float zmax, inv_den, fp;
+                            const float *zt = logits + (size_t)t * N;
+                            token_softmax_stats(zt, counts_slot, N, inv_T, zmax, inv_den, fp);
+                            for (int i = 0; i < 8; ++i)
+                                if (g0 + i < N)
+                                    v[i] += aux_scale * expf(zt[g0 + i] - zmax) * inv_den *
+                                            ((float)counts_slot[g0 + i] * inv_T - fp);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(v[i]);
+                    zh[i * kDwrZPitch + tl] = hi;
+                    zl[i * kDwrZPitch + tl] = __float2bfloat16_rn(v[i] - __bfloat162float(hi));
+                }
+            }
+            __syncwarp();
+            uint32_t af[4][4];                 // A fragments of the four 16-token steps
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                af[ks][0] = *reinterpret_cast<const uint32_t *>(zh + g * kDwrZPitch + 16 * ks + 2 * tq);
+                af[ks][1] = *reinterpret_cast<const uint32_t *>(zl + g * kDwrZPitch + 16 * ks + 2 * tq);
+                af[ks][2] = *reinterpret_cast<const uint32_t *>(zh + g * kDwrZPitch + 16 * ks + 2 * tq + 8);
+                af[ks][3] = *reinterpret_cast<const uint32_t *>(zl + g * kDwrZPitch + 16 * ks + 2 * tq + 8);
+            }
+            // rows lane / 4 + 8 i of the staged chunk, 16-byte piece lane % 4
+            auto fetch = [&](int c0, uint4 (&buf)[8]) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = (lane >> 2) + 8 * i;
+                    buf[i] = (r < ntok && c0 < c_end)
+                                 ? *reinterpret_cast<const uint4 *>(x + (size_t)(t0 + r) * d + c0 + (lane & 3) * 8)
+                                 : make_uint4(0u, 0u, 0u, 0u);
+                }
+            };
+            uint4 cur[8];
+            fetch(c_begin, cur);
+            for (int c0 = c_begin; c0 < c_end; c0 += kDwrChunkCols) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    *reinterpret_cast<uint4 *>(xs + ((lane >> 2) + 8 * i) * kDwrXPitch + (lane & 3) * 16) = cur[i];
+                __syncwarp();
+                fetch(c0 + kDwrChunkCols, cur);                   // the next chunk travels while this one is multiplied
+                float acc[4][4];
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+                    for (int np = 0; np < 2; ++np) {
+                        // matrix lane / 8: tokens 16 ks + 8 (m & 1) .., columns 16 np + 8 (m >> 1) ..
+                        const int m = lane >> 3;
+                        const uint32_t addr = xs_addr + (16 * ks + 8 * (m & 1) + (lane & 7)) * kDwrXPitch +
+                                              (16 * np + 8 * (m >> 1)) * 2;
+                        uint32_t b[4];
+                        ldmatrix_x4_trans(b, addr);
+                        mma_bf16_16816(acc[2 * np], af[ks][0], af[ks][1], af[ks][2], af[ks][3], b[0], b[1]);
+                        mma_bf16_16816(acc[2 * np + 1], af[ks][0], af[ks][1], af[ks][2], af[ks][3], b[2], b[3]);
+                    }
+                }
+                __syncwarp();                                     // the chunk has been read: it may be overwritten
+                if (g0 + g < N) {
+                    float *dst = dwr_partial + ((size_t)blk * N + g0 + g) * d + c0 + 2 * tq;
+#pragma unroll
+                    for (int nt = 0; nt < 4; ++nt)
+                        *reinterpret_cast<float2 *>(dst + nt * 8) =
+                            make_float2(acc[nt][0] + acc[nt][2], acc[nt][1] + acc[nt][3]);
+                }
+            }
+        }
+    }
+}
+
 // Sums the per-block partials in a fixed order: warp p of a block adds the partials b = p, p + 8, ... of 32
 // elements, then the eight warp sums are added in warp order.
 __global__ void __launch_bounds__(256)
@@ -1190,13 +1329,34 @@ cudaError_t launch_router_bwd(modse_dtype_t dt, const LayerMeta &m, const void *
     for (int pass = 0; pass < (noise ? 2 : 1); ++pass) {
         const float *dense = pass ? du : nullptr;
         const float ascale = pass ? 0.f : aux_scale;
-        if (dt == MODSE_F32)
+        if (dt == MODSE_F32) {
             router_dwr_kernel<float><<<grid, 256, 0, s>>>((const float *)x, T, m.d, m.N, m.k, p.topk_idx, p.dz,
                                                           p.dwr_partial, p.logits, p.counts_slot, ascale, dense);
-        else
+        } else if (m.d % kDwrChunkCols == 0) {
+            // tensor-core form: units of 64 tokens x 256 columns, one per warp, dealt round-robin to the blocks
+            const int nslice = (m.d + kDwrUnitCols - 1) / kDwrUnitCols;
+            const int units = nblk_dwr * nslice;
+            int dev = 0, sms = 0;
+            if (cudaGetDevice(&dev) != cudaSuccess ||
+                cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+                sms = 148;
+            const int grid_mma = std::max(1, std::min(units, 2 * sms));     // two blocks of 118 registers x 256 threads per SM
+            const size_t smem = (size_t)8 * kDwrWarpSmem;
+            static bool attr_done = false;
+            if (!attr_done) {
+                cudaError_t e = cudaFuncSetAttribute(router_dwr_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     (int)smem);
+                if (e != cudaSuccess) return e;
+                attr_done = true;
+            }
+            router_dwr_mma_kernel<<<grid_mma, 256, smem, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k, p.topk_idx, p.dz,
+                                                             p.dwr_partial, p.logits, p.counts_slot, ascale, dense,
+                                                             nblk_dwr, nslice);
+        } else {
             router_dwr_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, T, m.d, m.N, m.k,
                                                                   p.topk_idx, p.dz, p.dwr_partial, p.logits,
                                                                   p.counts_slot, ascale, dense);
+        }
         MODSE_LAUNCH_CHECK();
         reduce_dwr_kernel<<<(n + 31) / 32, 256, 0, s>>>(p.dwr_partial, nblk_dwr, n, pass ? ng.dw_noise : dw_router);
         MODSE_LAUNCH_CHECK();
