@@ -59,7 +59,10 @@ WsLayout make_layout(const LayerMeta &m, const int *h_desc, int esz, int T, bool
         return o;
     };
     const size_t kT = (size_t)m.k * T, N = m.N;
-    L.status = take(64);
+    // head: status word and tile counters (64 bytes), then the router's histogram sums per super-block, which it
+    // adds into: one cudaMemsetAsync zeroes both
+    L.head_bytes = 64 + (size_t)((L.nblk + kSuperBlocks - 1) / kSuperBlocks) * m.k * N * 4;
+    L.status = take(L.head_bytes);
     L.topk_idx = take(kT * 4);
     L.topk_gate = take(kT * 4);
     L.counts = take(N * 4);
@@ -120,6 +123,7 @@ WsPtrs carve(void *ws, const WsLayout &L)
     p.ptoken_of = (int *)(b + L.ptoken_of);
     p.pgate = (float *)(b + L.pgate);
     p.block_counts = (int *)(b + L.block_counts);
+    p.super_counts = (int *)(b + L.status + 64);
     p.logits = (float *)(b + L.logits);
     p.aux_partial = (float *)(b + L.aux_partial);
     p.noise_u = (float *)(b + L.noise_u);
@@ -349,7 +353,7 @@ modse_status_t modse_forward(modse_layer_t *layer, modse_dtype_t dtype, const mo
     const int fuse = effective_fuse(layer, dtype, of32);
 
     StageTimer tm(layer, s);
-    MODSE_CUDA(cudaMemsetAsync(p.status, 0, 64, s));           // status word and the tile counters
+    MODSE_CUDA(cudaMemsetAsync(p.status, 0, L.head_bytes, s));   // status word, tile counters, super-block sums
     if (layer->debug_checks) MODSE_CUDA(launch_canaries(workspace, L, false, p.status, s));
     MODSE_STAGE(tm, 0, launch_router(dtype, m, x, weights->w_router, n_tokens, p, layer->noise, s, &launches));
     MODSE_STAGE(tm, 1, launch_rank(m, n_tokens, L.Pmax, p, s, &launches));

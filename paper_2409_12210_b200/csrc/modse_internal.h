@@ -14,12 +14,14 @@ namespace modse {
 constexpr int kMaxExperts = 256;
 constexpr int kRowPad = 128;        // every expert group is padded to a multiple of this many rows
 constexpr int kRouterTokB = 64;     // tokens per block in the router / rank kernels
+constexpr int kSuperBlocks = 32;    // router blocks per super-block (the router also keeps histogram sums per super-block)
 constexpr int kRouterBwdTokB = 128; // tokens per block in the router backward kernel
 constexpr int kDwrTokB = 64;        // tokens per partial sum of dW_router = dz^T x
 constexpr int kPanel = 64;          // hidden-axis panel width of the bf16 activation layout
 
 // Device status word values (first int of the workspace).  Ints 4..9 of the same 64-byte block are the
-// tile counters of the six grouped products (zeroed with it).
+// tile counters of the six grouped products (zeroed with it); the router's histogram sums per super-block
+// (super_counts) follow the block directly and are zeroed by the same call.
 enum : int { kDevOk = 0, kDevTimeout = 1, kDevBounds = 2 };
 
 // Every workspace region is followed by a 256-byte guard block.  With the debug checks on its first 8 bytes
@@ -37,6 +39,7 @@ struct LayerMeta {
 struct WsLayout {
     int T, R, Pmax, nblk, nblk_bwd;
     size_t hb;   // element capacity of each [padded rows x h_e] activation buffer
+    size_t head_bytes;   // status block + super_counts: what the start of a forward zeroes
     size_t status, topk_idx, topk_gate, counts, counts_slot, offsets, poffsets, ebase, row_of, token_of,
         prow_of, ptoken_of, pgate, block_counts, logits, aux_partial, noise_u, du, dgamma_partial, dg, dz, dwr_partial, xp, a_pre, b_pre, hm, o, dyp, da, db, dxp,
         dg_part, total;
@@ -54,6 +57,7 @@ struct WsPtrs {
     int *row_of, *token_of, *prow_of, *ptoken_of;
     float *pgate;
     int *block_counts;
+    int *super_counts;   // [ceil(nblk / kSuperBlocks)][k*N] sums of block_counts over super-blocks
     float *logits;       // [T,N] router logits (may be null: not stored)
     float *aux_partial;  // [nblk_bwd][N] partial sums of the router probabilities
     float *noise_u;      // [T,N] x W_n, kept for the backward of the second term of Eq. 2

@@ -36,7 +36,7 @@ ScratchLayout scratch_layout(int T, int N, int k, int Pmax, int nblk)
     ScratchLayout L{};
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    L.status = take(64);
+    L.status = take(64 + (size_t)((nblk + modse::kSuperBlocks - 1) / modse::kSuperBlocks) * k * N * 4);   // status, then super-block sums
     L.poffsets = take((size_t)(N + 1) * 4);
     L.ebase = take((size_t)(N + 1) * 8);
     L.prow_of = take((size_t)k * T * 4);
@@ -99,6 +99,7 @@ extern "C" modse_status_t modse_route_static_scratch(modse_dtype_t dtype, int d_
     p.ptoken_of = reinterpret_cast<int *>(base + L.ptoken_of);
     p.pgate = reinterpret_cast<float *>(base + L.pgate);
     p.block_counts = reinterpret_cast<int *>(base + L.block_counts);
+    p.super_counts = reinterpret_cast<int *>(base + L.status + 64);
     p.logits = nullptr;                             // the logits themselves are not kept
     p.topk_idx = topk_idx;
     p.topk_gate = topk_gate;
@@ -109,9 +110,10 @@ extern "C" modse_status_t modse_route_static_scratch(modse_dtype_t dtype, int d_
     p.token_of = token_of;
 
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    // the array keeps the previous call's bytes: the status word must start at zero, every
-    // other region is fully rewritten by the two kernels before it is read
-    if (cudaMemsetAsync(p.status, 0, 64, s) != cudaSuccess) return MODSE_ERR_CUDA;
+    // the array keeps the previous call's bytes: the status word and the super-block sums the router adds into
+    // must start at zero, every other region is fully rewritten by the two kernels before it is read
+    const size_t head = 64 + (size_t)((nblk + kSuperBlocks - 1) / kSuperBlocks) * top_k * n_experts * 4;
+    if (cudaMemsetAsync(p.status, 0, head, s) != cudaSuccess) return MODSE_ERR_CUDA;
     if (launch_router(dtype, m, x, w_router, n_tokens, p, NoiseGate{}, s, nullptr) != cudaSuccess) return MODSE_ERR_CUDA;
     if (launch_rank(m, n_tokens, Pmax, p, s, nullptr) != cudaSuccess) return MODSE_ERR_CUDA;
     return MODSE_OK;

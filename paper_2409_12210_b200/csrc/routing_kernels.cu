@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(256)
 router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok, int d, int N, int k,
               int *__restrict__ topk_idx, float *__restrict__ topk_gate, int *__restrict__ block_counts,
               float *__restrict__ logits, int w_in_smem, const T *__restrict__ w_noise, float gamma, float eps,
-              float *__restrict__ noise_u)
+              float *__restrict__ noise_u, int *__restrict__ super_counts)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int Npad = (N + 3) & ~3;
@@ -206,7 +206,13 @@ router_kernel(const T *__restrict__ x, const T *__restrict__ w_router, int Ttok,
         __syncwarp();
     }
     __syncthreads();
-    for (int i = tid; i < k * N; i += blockDim.x) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
+    // the block's histogram, and its share of the sums over super-blocks of kSuperBlocks blocks (integer
+    // atomics into words zeroed with the status word: the result does not depend on their order)
+    for (int i = tid; i < k * N; i += blockDim.x) {
+        const int c = cnt[i];
+        block_counts[(size_t)blockIdx.x * k * N + i] = c;
+        if (c != 0) atomicAdd(&super_counts[(size_t)(blockIdx.x / kSuperBlocks) * k * N + i], c);
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -247,7 +253,8 @@ __global__ void __launch_bounds__(kRouterMmaThreads, 2)      // two 512-thread b
 router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__restrict__ w_router, int Ttok, int d,
                   int N, int k, int *__restrict__ topk_idx, float *__restrict__ topk_gate,
                   int *__restrict__ block_counts, float *__restrict__ logits,
-                  const __nv_bfloat16 *__restrict__ w_noise, float gamma, float eps, float *__restrict__ noise_u)
+                  const __nv_bfloat16 *__restrict__ w_noise, float gamma, float eps, float *__restrict__ noise_u,
+                  int *__restrict__ super_counts)
 {
     constexpr int NTT = NOISE ? 2 * NT : NT;            // n-tiles accumulated per warp
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -406,17 +413,23 @@ router_mma_kernel(const __nv_bfloat16 *__restrict__ x, const __nv_bfloat16 *__re
         }
     }
     __syncthreads();
-    for (int i = tid; i < k * N; i += kRouterMmaThreads) block_counts[(size_t)blockIdx.x * k * N + i] = cnt[i];
+    for (int i = tid; i < k * N; i += kRouterMmaThreads) {
+        const int c = cnt[i];
+        block_counts[(size_t)blockIdx.x * k * N + i] = c;
+        if (c != 0) atomicAdd(&super_counts[(size_t)(blockIdx.x / kSuperBlocks) * k * N + i], c);
+    }
 }
 
 // ---------------------------------------------------------------------------
 // Rank: block b owns tokens [b*64, b*64+64).  It sums the histograms of the
-// blocks before it (tokens before its own), scans the totals over experts, and
-// ranks its own assignments by token index.  Integer work only.
+// blocks before it (tokens before its own) - whole super-blocks of 32 blocks from
+// the sums the router kept, then the blocks of its own super-block -, scans the
+// totals over experts, and ranks its own assignments by token index.  Integer
+// work only.
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 rank_kernel(LayerMeta m, int Ttok, int Pmax, int nblk, const int *__restrict__ block_counts,
-            const int *__restrict__ topk_idx, const float *__restrict__ topk_gate, int *__restrict__ counts,
+            const int *__restrict__ super_counts, const int *__restrict__ topk_idx, const float *__restrict__ topk_gate, int *__restrict__ counts,
             int *__restrict__ counts_slot, int *__restrict__ offsets, int *__restrict__ poffsets,
             long long *__restrict__ ebase, int *__restrict__ row_of, int *__restrict__ token_of,
             int *__restrict__ prow_of, int *__restrict__ ptoken_of, float *__restrict__ pgate, int *status)
@@ -436,25 +449,30 @@ rank_kernel(LayerMeta m, int Ttok, int Pmax, int nblk, const int *__restrict__ b
     for (int p = tid; p < 2 * kN; p += 256) tot[p] = 0;       // tot and pre are adjacent
     __syncthreads();
     {
+        // sums over whole super-blocks (all of them for the totals, those before this block's for its prefix),
+        // then the blocks of this block's own super-block that lie before it
+        const int nsb = (nblk + kSuperBlocks - 1) / kSuperBlocks, sb = b / kSuperBlocks;
         const int groups = max(1, 256 / kN);
         const int gidx = tid / kN, p = tid % kN;
         if (gidx < groups && tid < 256) {
             int before = 0, all = 0;
-            for (int bb = gidx; bb < nblk; bb += groups) {
-                const int c = block_counts[(size_t)bb * kN + p];
+            for (int s2 = gidx; s2 < nsb; s2 += groups) {
+                const int c = super_counts[(size_t)s2 * kN + p];
                 all += c;
-                if (bb < b) before += c;
+                if (s2 < sb) before += c;
             }
+            for (int bb = sb * kSuperBlocks + gidx; bb < b; bb += groups) before += block_counts[(size_t)bb * kN + p];
             atomicAdd(&tot[p], all);
             atomicAdd(&pre[p], before);
         }
         for (int q = 256 + tid; q < kN; q += 256) {            // more pairs than threads: the rest, one thread each
             int before = 0, all = 0;
-            for (int bb = 0; bb < nblk; ++bb) {
-                const int c = block_counts[(size_t)bb * kN + q];
+            for (int s2 = 0; s2 < nsb; ++s2) {
+                const int c = super_counts[(size_t)s2 * kN + q];
                 all += c;
-                if (bb < b) before += c;
+                if (s2 < sb) before += c;
             }
+            for (int bb = sb * kSuperBlocks; bb < b; ++bb) before += block_counts[(size_t)bb * kN + q];
             tot[q] = all;
             pre[q] = before;
         }
@@ -1167,7 +1185,7 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
             if (e != cudaSuccess) return e;
             kern<<<nblk, kRouterMmaThreads, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
                                          p.topk_idx, p.topk_gate, p.block_counts, p.logits,
-                                         (const __nv_bfloat16 *)ng.w_noise, ng.gamma, ng.eps, p.noise_u);
+                                         (const __nv_bfloat16 *)ng.w_noise, ng.gamma, ng.eps, p.noise_u, p.super_counts);
             MODSE_LAUNCH_CHECK();
             return cudaSuccess;
         }
@@ -1183,14 +1201,14 @@ cudaError_t launch_router(modse_dtype_t dt, const LayerMeta &m, const void *x, c
         if (e != cudaSuccess) return e;
         kern<<<nblk, 256, smem, s>>>((const float *)x, (const float *)w_router, T, m.d, m.N, m.k, p.topk_idx,
                                      p.topk_gate, p.block_counts, p.logits, w_in_smem, (const float *)ng.w_noise,
-                                     ng.gamma, ng.eps, p.noise_u);
+                                     ng.gamma, ng.eps, p.noise_u, p.super_counts);
     } else {
         auto kern = router_kernel<__nv_bfloat16>;
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         kern<<<nblk, 256, smem, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w_router, T, m.d, m.N, m.k,
                                      p.topk_idx, p.topk_gate, p.block_counts, p.logits, w_in_smem,
-                                     (const __nv_bfloat16 *)ng.w_noise, ng.gamma, ng.eps, p.noise_u);
+                                     (const __nv_bfloat16 *)ng.w_noise, ng.gamma, ng.eps, p.noise_u, p.super_counts);
     }
     MODSE_LAUNCH_CHECK();
     return cudaSuccess;
@@ -1201,7 +1219,7 @@ cudaError_t launch_rank(const LayerMeta &m, int T, int Pmax, const WsPtrs &p, cu
     const int nblk = (T + kRouterTokB - 1) / kRouterTokB;
     const int kN = m.k * m.N;
     const size_t smem = sizeof(int) * (2 * kN + 2 * (m.N + 1) + m.N + kRouterTokB * m.k);
-    rank_kernel<<<nblk, 256, smem, s>>>(m, T, Pmax, nblk, p.block_counts, p.topk_idx, p.topk_gate, p.counts,
+    rank_kernel<<<nblk, 256, smem, s>>>(m, T, Pmax, nblk, p.block_counts, p.super_counts, p.topk_idx, p.topk_gate, p.counts,
                                         p.counts_slot, p.offsets, p.poffsets, p.ebase, p.row_of, p.token_of,
                                         p.prow_of, p.ptoken_of, p.pgate, p.status);
     MODSE_LAUNCH_CHECK();
