@@ -1,8 +1,8 @@
 // Grouped GEMMs of the bf16 MoDSE layer on Blackwell tensor cores.
 //
-// One persistent, warp-specialised kernel template serves the six products of
-// the layer (Sec. 3.1, Eq. 4 and its gradient); the accumulators (fp32) live in
-// tensor memory (TMEM):
+// Two persistent, warp-specialised kernel templates (one CTA per tile, or a pair
+// of CTAs per tile) serve the six products of the layer (Sec. 3.1, Eq. 4 and its
+// gradient); the accumulators (fp32) live in tensor memory (TMEM):
 //
 //   kind            product (per expert e, cp = padded rows, h = width)      K
 //   UpGate          Hm = g * silu(xp Wg^T) * (xp Wu^T)      [cp, h]          d
@@ -12,10 +12,13 @@
 //   UpGateDgrad     dxp = dA Wg_e + dB Wu_e                 [cp, d]  fp32    2h
 //   UpGateWgrad     dWg_e = dA^T xp, dWu_e = dB^T xp        [h, d]           cp
 //
-// Two tile shapes: 128 rows x up to 256 accumulator columns with two
+// Three tile shapes.  One CTA: 128 rows x up to 256 accumulator columns with two
 // accumulators in flight (the epilogue of one tile overlaps the main loop of the
-// next), and 256 rows (two 128-row halves that share the column operand, 2/3 of
+// next), or 256 rows (two 128-row halves that share the column operand, 2/3 of
 // the shared-memory traffic per FLOP, but both accumulators belong to one tile).
+// A pair of CTAs (cta_group::2, the default): 256 rows, each CTA stages its own
+// 128 rows and half of the column operand and holds its half of the accumulator
+// - the traffic of the second shape with the overlap of the first.
 //
 // Roles inside a CTA: warp 0 issues TMA loads into a ring of shared-memory
 // stages (boxes of 64 elements x 64 or 128 rows, 128-byte swizzle), warp 1
@@ -49,11 +52,11 @@
 //
 // Tile order: experts by decreasing K, so the long tiles of wide experts (or of
 // experts with many tokens) start first and the short ones fill the tail - the
-// one-GPU form of the paper's expert-pair balancing (Sec. 3.2).  CTAs take the
-// next tile of that list from a counter in global memory (or, with the
-// counter switched off, are dealt tiles round-robin).  Every output tile is
-// computed by one CTA with its K blocks in ascending order either way, so the
-// results do not depend on which CTA ran which tile.  The counter is read by a
+// one-GPU form of the paper's expert-pair balancing (Sec. 3.2).  CTAs (or CTA
+// pairs) take the next tile of that list from a counter in global memory (or,
+// with the counter switched off, are dealt tiles round-robin).  Every output
+// tile is computed by one CTA or one pair with its K blocks in ascending order
+// either way, so the results do not depend on who ran which tile.  The counter is read by a
 // warp of its own, which passes the tile indices to the three working roles
 // through a small queue in shared memory: an atomic instruction inside the
 // loop of the thread that issues the TMA loads cost the 128-row kernels a
