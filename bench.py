@@ -250,8 +250,11 @@ def main():
                          "default benchmark, whose router is x W_g alone")
     ap.add_argument("--aux-alpha", type=float, default=0.0,
                     help="coefficient of the auxiliary load-balance loss (Eq. 7) added to the objective in backward")
-    ap.add_argument("--no-tune", action="store_true",
-                    help="skip the set-up call that times the kernel shapes of the forward products on this GPU")
+    ap.add_argument("--tune", action="store_true",
+                    help="set-up: let modse_tune_forward time the kernel shapes of the forward products on this GPU "
+                         "(off by default: the library's default plan, CTA pairs everywhere, was the faster one inside "
+                         "a forward + backward step on every board measured)")
+    ap.add_argument("--no-tune", action="store_true", help="accepted and ignored: not tuning is the default")
     ap.add_argument("--no-equal-size", action="store_true",
                     help="skip the interleaved comparison with the equal-size layer of the same total width")
     ap.add_argument("--skew-pair", action="store_true",
@@ -303,7 +306,7 @@ def main():
     T, d, K, W = cfg.n_tokens, cfg.d_model, args.steps, max(args.warmup, 3)
     L = max(1, args.layers)
     do_bwd = cfg.backward
-    tune = dt == torch.bfloat16 and not args.no_tune and args.tile_plan is None
+    tune = dt == torch.bfloat16 and args.tune and args.tile_plan is None
 
     class Replica:
         """One layer with all its tensors resident on the device.  `host` holds seeded host tensors (the

@@ -192,11 +192,14 @@ modse_status_t modse_set_output_f32(modse_layer_t *layer, int on);
 /* Choice of kernel shape per device (no counterpart in the paper: a property of this implementation).
  * Each grouped product of the bf16 layer exists with 128-row tiles, with 256-row tiles computed by one CTA and
  * with 256-row tiles computed by a pair of CTAs; which is fastest for the two forward products depends on how
- * fast the GPU at hand feeds shared memory from L2, which differs between otherwise identical boards.  modse_tune_forward runs the forward pass (arguments as modse_forward) a few
- * times per candidate on the caller's own buffers, times it with CUDA events, and keeps the fastest plan in
+ * fast the GPU at hand feeds shared memory from L2, which differs between otherwise identical boards.
+ * modse_tune_forward runs the forward pass (arguments as modse_forward) a few times per candidate on the caller's own buffers, times it with CUDA events, and keeps the fastest plan in
  * the layer object for all later calls.  It allocates no device memory, SYNCHRONISES the stream, and leaves y
  * and the workspace as one modse_forward would.  Results do not depend on the plan (the K order of every sum
  * is the same).  fp32 layers have one kernel shape: the call returns MODSE_OK at once.
+ * The plan it finds is the fastest for forward passes run on their own (serving); inside a training step the
+ * stages share the GPU's power budget and the library default (CTA pairs for every product) has been the faster
+ * choice on every board measured, so training code need not call it.
  * modse_get_tile_plan returns the plan: -1 for the library default, else a bit set with, for product k (0 up/gate,
  * 1 down, 2 down dgrad, 3 down wgrad, 4 up/gate dgrad, 5 up/gate wgrad), bit 8 + k set: 256-row tiles computed
  * by a pair of CTAs on neighbouring SMs; otherwise bit k set: 256-row tiles computed by one CTA, clear: 128-row
