@@ -1165,8 +1165,17 @@ reduce_dwr_kernel(const float *__restrict__ partial, int nblk, int n, float *__r
     const int lane = threadIdx.x & 31, p = threadIdx.x >> 5;
     const int i = blockIdx.x * 32 + lane;
     float s = 0.f;
-    if (i < n)
-        for (int b = p; b < nblk; b += 8) s += partial[(size_t)b * n + i];
+    if (i < n) {
+        // eight loads in flight at a time; the additions keep their order
+        for (int b0 = p; b0 < nblk; b0 += 64) {
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = b0 + 8 * u < nblk ? partial[(size_t)(b0 + 8 * u) * n + i] : 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (b0 + 8 * u < nblk) s += v[u];
+        }
+    }
     part[p][lane] = s;
     __syncthreads();
     if (p == 0 && i < n) {
