@@ -42,9 +42,9 @@ BURST_REGION_S = 1.0                   # timed regions shorter than this run on 
 # valid only for that workload, for the library's default tile plan and for the kernel source they were taken
 # from (first 16 hex digits of the SHA-256 of csrc/tc_gemm.cu), otherwise "traffic" is reported as null.
 NCU_TRAFFIC = {
-    "workload": "train_16k", "tc_gemm_sha256_16": "89218d4718a93511",
-    "bytes_per_launch": {"upgate_gemm_swiglu": 1.589e9, "down_gemm": 0.948e9, "down_dgrad_swiglu_bwd": 1.831e9,
-                         "down_wgrad": 0.686e9, "upgate_dgrad": 1.910e9, "upgate_wgrad": 1.242e9},
+    "workload": "train_16k", "tc_gemm_sha256_16": "4025bd8c15f9c71a",
+    "bytes_per_launch": {"upgate_gemm_swiglu": 1.592e9, "down_gemm": 1.022e9, "down_dgrad_swiglu_bwd": 1.849e9,
+                         "down_wgrad": 0.688e9, "upgate_dgrad": 1.976e9, "upgate_wgrad": 1.244e9},
 }
 
 

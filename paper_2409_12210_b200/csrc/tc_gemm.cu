@@ -1598,6 +1598,7 @@ EncodeTiledFn get_encode()
 }
 
 // bf16 row-major matrix [rows, cols] seen as a 2-D tensor, boxes of box_cols columns x box_rows rows.
+// L2 promotion of 128 bytes: measured 1.5-2 % faster per step than 256 bytes or none (two alternating runs each).
 bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows = 64,
                uint32_t box_cols = 64, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B)
 {
@@ -1608,7 +1609,7 @@ bool encode_2d(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols,
     const cuuint32_t box[2] = {box_cols, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
