@@ -546,6 +546,10 @@ def main():
     ms_e2e = ev0.elapsed_time(ev1)
     ms_e2e = max_over_ranks(ms_e2e, dev)
     e2e_value = whole_job_value(T, world, ms_e2e / K)
+    # no kernel of any timed region may have given up a wait or met a bad index: the numbers would mean nothing
+    status = layer.check_device_status(ws)
+    if status != 0:
+        raise SystemExit(f"device status {status} after the timed regions: {B.status_string(status)}")
 
     if rank != 0:
         if world > 1:
